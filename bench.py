@@ -1,0 +1,464 @@
+#!/usr/bin/env python
+"""Benchmark of the WeDLM decoding step (reorder -> window attention -> confidence/commit).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3_batched] [--attn auto]
+    python bench.py --impl reference ...        # the fp64 CPU oracle on a bounded sample
+
+One "step" is one pass of the whole hot path over one batch of seeded synthetic inputs.  With
+N > 1 (launched under torchrun) every rank runs the same-shaped batch drawn from its own seed
+(weak scaling, sequences are independent: no collective on the data path) and rank 0 prints the
+aggregate.  Prints ONE JSON line on stdout; progress goes to stderr.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "committed_tokens_per_s"
+UNIT = "tokens/s"
+L2_BYTES = 126 * 1024 * 1024
+
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from
+# one ncu capture; the summaries under profiles/ give the commands).  None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while the GPU works."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, device_index: int, period_s: float = 0.002):
+        self.samples = []          # (t, sm_mhz, reasons_mask, tag)
+        self.tag = "idle"
+        self.period = period_s
+        self._stop = threading.Event()
+        self.ok = False
+        self.max_mhz = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as e:          # pragma: no cover - depends on the box
+            log("clock sampling unavailable:", repr(e))
+        self.thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                self.samples.append((time.time(), mhz, mask, self.tag))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.ok:
+            self.thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self.ok and self.thread.is_alive():
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        timed = [s for s in self.samples if s[3] == "timed"]
+        use = timed if len(timed) >= 3 else [s for s in self.samples if s[3] != "idle"]
+        if not use:
+            use = self.samples
+        mask = 0
+        for s in use:
+            mask |= s[2]
+        reasons = [name for bit, name in self.REASONS.items() if mask & bit]
+        return {"sm_mhz": statistics.median(s[1] for s in use), "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(use), "samples_in_timed_region": len(timed)}
+
+
+# ----------------------------------------------------------------------------------------------
+# workload helpers
+# ----------------------------------------------------------------------------------------------
+def algorithmic_bytes(cfg, inp):
+    """Bytes the method itself must move per step (one layer)."""
+    elem = 2 if cfg.dtype == "bf16" else 4
+    B, W = inp["filled"].shape
+    kv_tokens = int(inp["prefix_len"].astype(np.int64).sum()) + B * W
+    kv = kv_tokens * cfg.n_kv_heads * cfg.head_dim * 2 * elem             # K and V, prefix + window rows
+    q_io = 2 * B * W * cfg.n_q_heads * cfg.head_dim * elem                # rotated q read + out write
+    n_mask_rows = int((inp["filled"] == 0).sum())
+    logits = n_mask_rows * cfg.vocab * elem
+    return {"attn_kernel": kv + q_io, "kv_stream": kv, "logits_stream": logits, "mask_rows": n_mask_rows}
+
+
+def slice_batch(inp, n):
+    out = {}
+    for k, v in inp.items():
+        out[k] = v if k in ("k_cache", "v_cache") else v[:n]
+    return out
+
+
+def oracle_step_time(cfg, inp, n_seqs):
+    from oracle import wedlm_oracle as orc
+    sub = slice_batch(inp, n_seqs)
+    t0 = time.perf_counter()
+    r = orc.step(sub, theta=cfg.rope_theta, conf_mode=cfg.conf_mode, tau=cfg.tau, lam=cfg.lam,
+                 maxprob_thr=cfg.maxprob_thr, mask_token_id=cfg.mask_token_id, page_size=cfg.page_size)
+    dt = time.perf_counter() - t0
+    committed = int(sum(ps["committed_count"] for ps in r["per_seq"]))
+    return dt, committed
+
+
+# ----------------------------------------------------------------------------------------------
+# reference arm: the oracle on host cores
+# ----------------------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from workloads import get_config, make_step, BASE_SEED
+    cfg = get_config(args.workload)
+    inp = make_step(cfg, seed=BASE_SEED)
+    cores = len(os.sched_getaffinity(0))
+    # size the per-step sample so that the whole run stays within a few minutes
+    t1, _ = oracle_step_time(cfg, inp, 1)
+    budget_s = 150.0
+    n = int(max(1, min(cfg.batch, budget_s / max(t1, 1e-3) / (args.steps + args.warmup))))
+    for _ in range(args.warmup):
+        oracle_step_time(cfg, inp, n)
+    times, committed = [], 0
+    for _ in range(args.steps):
+        dt, c = oracle_step_time(cfg, inp, n)
+        times.append(dt)
+        committed = c
+    total = sum(times)
+    value = committed * args.steps / total if total > 0 else 0.0
+    sample = f"first {n} of {cfg.batch} sequences of {cfg.name} per step (all heads, all mask rows)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ----------------------------------------------------------------------------------------------
+# product arm
+# ----------------------------------------------------------------------------------------------
+class Workload:
+    """Device-resident inputs of one workload, with `n_copies` rotating copies of the large
+    streams (cache, logits) when one copy would fit in L2, and one fresh copy of the small window
+    state per iteration."""
+
+    def __init__(self, name, seed, attn_impl, n_state):
+        import torch
+        import paper_2512_22737_b200 as w
+        from workloads import get_config, make_step
+        self.cfg = get_config(name)
+        t0 = time.time()
+        self.inp = make_step(self.cfg, seed=seed)
+        log(f"[{name}] inputs drawn in {time.time() - t0:.1f}s")
+        inp = self.inp
+        self.bytes = algorithmic_bytes(self.cfg, inp)
+        big = inp["k_cache"].nbytes + inp["v_cache"].nbytes + inp["logits"].nbytes
+        self.n_copies = 1 if big > 2 * L2_BYTES else int(np.ceil(3 * L2_BYTES / big)) + 1
+        self.c = w.config_for(self.cfg, max_pages_per_seq=inp["block_table"].shape[1],
+                              num_pages=inp["k_cache"].shape[0], max_prefix_len=int(inp["prefix_len"].max()),
+                              attn_impl=attn_impl)
+        self.step = w.DecodeStep(self.c)
+        self.static = {k: w.to_device(inp[k]) for k in ("q", "k", "v", "block_table")}
+        self.big = [{k: (w.to_device(inp[k]) if i == 0 else None) for k in ("k_cache", "v_cache", "logits")}
+                    for i in range(self.n_copies)]
+        for i in range(1, self.n_copies):
+            for k in ("k_cache", "v_cache", "logits"):
+                self.big[i][k] = self.big[0][k].clone()
+        self.state0 = {k: w.to_device(inp[k]) for k in ("filled", "window_tokens", "prefix_len")}
+        self.states = [{k: v.clone() for k, v in self.state0.items()} for _ in range(n_state)]
+        self.it = 0
+        self.committed_per_step = None
+        torch.cuda.synchronize()
+
+    def reset_states(self):
+        for s in self.states:
+            for k, v in self.state0.items():
+                s[k].copy_(v)
+        self.it = 0
+
+    def run_step(self, profile_events=None):
+        import paper_2512_22737_b200 as w
+        big = self.big[self.it % self.n_copies]
+        st = self.states[self.it % len(self.states)]
+        self.it += 1
+        d = dict(self.static)
+        d.update(big)
+        d.update(st)
+        s = self.step
+        s.reorder(d["filled"], d["window_tokens"], d["prefix_len"])
+        if profile_events is not None:
+            w.wedlm_profile_next_attn(*profile_events)
+        s.attention(d["q"], d["k"], d["v"], d["k_cache"], d["v_cache"], d["block_table"], d["prefix_len"])
+        s.confidence_commit(d["logits"], d["window_tokens"], d["filled"], d["prefix_len"])
+
+
+def time_workload(wl, steps, warmup, sampler=None, tag="timed"):
+    """warmup + `steps` timed iterations; returns (ms_per_step, attn_kernel_ms_avg, committed, launches)."""
+    import torch
+    import paper_2512_22737_b200 as w
+    wl.reset_states()
+    for _ in range(warmup):
+        wl.run_step()
+    torch.cuda.synchronize()
+    committed = int(wl.step.committed_count.sum().item())
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:       # create the handles outside the timed region
+        a.record()
+        b.record()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = w.wedlm_launch_count()
+    if sampler:
+        sampler.tag = tag
+    start.record()
+    for i in range(steps):
+        wl.run_step(profile_events=evs[i])
+    stop.record()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.tag = "other"
+    launches = w.wedlm_launch_count() - l0
+    ms = start.elapsed_time(stop) / steps
+    attn_ms = sum(a.elapsed_time(b) for a, b in evs) / steps
+    return ms, attn_ms, committed, launches
+
+
+def time_e2e(wl, steps, warmup, sampler=None):
+    """The same step fed from pinned HOST buffers: every iteration copies the step's inputs (window
+    state, block table, q/k/v, logits) to the device, runs the three calls, and reads the commit
+    results back.  The KV cache is resident device state, as in a serving engine."""
+    import torch
+    inp = wl.inp
+    names = ["filled", "window_tokens", "prefix_len", "block_table", "q", "k", "v", "logits"]
+    host = {}
+    for k in names:
+        a = inp[k]
+        t = torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a)
+        host[k] = t.pin_memory()
+    dev = {k: torch.empty_like(host[k], device="cuda") for k in names}
+    view = {k: (dev[k].view(torch.bfloat16) if inp[k].dtype == np.uint16 else dev[k]) for k in names}
+    s = wl.step
+    out_host = {k: torch.empty_like(getattr(s, k), device="cpu").pin_memory()
+                for k in ("committed_count", "committed_tokens", "filled_count")}
+    h2d = sum(host[k].numel() * host[k].element_size() for k in names)
+    d2h = sum(v.numel() * v.element_size() for v in out_host.values())
+    big = wl.big[0]
+
+    def one():
+        for k in names:
+            dev[k].copy_(host[k], non_blocking=True)
+        s.reorder(view["filled"], view["window_tokens"], view["prefix_len"])
+        s.attention(view["q"], view["k"], view["v"], big["k_cache"], big["v_cache"], view["block_table"], view["prefix_len"])
+        s.confidence_commit(view["logits"], view["window_tokens"], view["filled"], view["prefix_len"])
+        for k, v in out_host.items():
+            v.copy_(getattr(s, k), non_blocking=True)
+
+    for _ in range(warmup):
+        one()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if sampler:
+        sampler.tag = "e2e"
+    start.record()
+    for _ in range(steps):
+        one()
+    stop.record()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.tag = "other"
+    ms = start.elapsed_time(stop) / steps
+    committed = int(out_host["committed_count"].sum().item())
+    return ms, committed, h2d, d2h
+
+
+def run_product(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2512_22737_b200 import build as b
+    from workloads import BASE_SEED
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        b.build()
+    if world > 1:
+        dist.barrier()
+    import paper_2512_22737_b200 as w
+    w.load_library()
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    n_state = args.steps + args.warmup
+    wl = Workload(args.workload, BASE_SEED + rank, args.attn, n_state)
+    if sampler:
+        sampler.start()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    barrier()
+    ms, attn_ms, committed, launches = time_workload(wl, args.steps, args.warmup, sampler)
+    barrier()
+    t = torch.tensor([ms, attn_ms, float(committed)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        tmax = t.clone()
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        tsum = t.clone()
+        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+        ms, attn_ms, committed_total = float(tmax[0]), float(tmax[1]), float(tsum[2])
+    else:
+        committed_total = float(committed)
+    assert int(wl.step.status.item()) == 0, "device status word set during the benchmark"
+
+    e2e_ms, e2e_committed, h2d, d2h = time_e2e(wl, max(3, min(args.steps, 10)), 3, sampler)
+    te = torch.tensor([e2e_ms, float(e2e_committed)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        tm = te.clone()
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        tsu = te.clone()
+        dist.all_reduce(tsu, op=dist.ReduceOp.SUM)
+        e2e_ms, e2e_committed = float(tm[0]), float(tsu[1])
+
+    others = {}
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_extras:
+        for name in ("cfg2_qwen_b1", "cfg4_long"):
+            if name == args.workload:
+                continue
+            try:
+                o = Workload(name, BASE_SEED, args.attn, n_state)
+                oms, oattn, ocommit, _ = time_workload(o, args.steps, args.warmup, sampler, tag="other")
+                ob = o.bytes
+                others[name] = {
+                    "ms_per_step": oms, "committed_tokens_per_s": ocommit / (oms * 1e-3),
+                    "attn_kernel_ms": oattn, "attn_kernel_GBps": ob["attn_kernel"] / (oattn * 1e-3) / 1e9,
+                    "rotating_copies": o.n_copies,
+                }
+                del o
+                torch.cuda.empty_cache()
+            except Exception as e:      # pragma: no cover
+                others[name] = {"error": repr(e)}
+    if sampler:
+        sampler.stop()
+    if rank == 0 and world == 1:
+        cores = len(os.sched_getaffinity(0))
+        n_s = min(wl.cfg.batch, 8 if wl.cfg.batch >= 8 else wl.cfg.batch)
+        log(f"timing the oracle on {n_s} sequences ...")
+        dt, c = oracle_step_time(wl.cfg, wl.inp, n_s)
+        cpu = {"value": c / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"one step over the first {n_s} of {wl.cfg.batch} sequences of {wl.cfg.name} "
+                         f"({dt:.1f}s of CPU wall time)"}
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        bts = wl.bytes
+        achieved = bts["attn_kernel"] / (attn_ms * 1e-3) / 1e9
+        key = f"{wl.cfg.name}:{args.attn}"
+        line = {
+            "metric": METRIC, "value": committed_total / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.cfg.dtype == "bf16" else "f32",
+            "data": "synthetic",
+            "config": {"workload": wl.cfg.name, "batch_per_gpu": wl.cfg.batch, "window": wl.cfg.window,
+                       "prefix_tokens_per_gpu": int(wl.inp["prefix_len"].sum()), "attn_impl": args.attn,
+                       "l2": "inputs_exceed_l2" if wl.n_copies == 1 else f"rotating_{wl.n_copies}_copies",
+                       "committed_tokens_per_step": committed_total,
+                       "kv_stream_bytes": bts["kv_stream"], "logits_stream_bytes": bts["logits_stream"]},
+            "clocks": sampler.summary() if sampler else None,
+            "e2e": {"value": e2e_committed / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "kernel": "window attention", "achieved": achieved, "peak": peak,
+                         "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                         "frac_of_nominal_8TBps": achieved / 8000.0,
+                         "traffic": NCU_TRAFFIC_BYTES.get(key), "kernel_ms": attn_ms,
+                         "algorithmic_bytes": bts["attn_kernel"]},
+            "cpu_baseline": cpu,
+            "other_workloads": others,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="product", choices=["product", "reference"])
+    ap.add_argument("--workload", default="cfg3_batched")
+    ap.add_argument("--attn", default="auto", choices=["auto", "generic", "tensor"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "product" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_product(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

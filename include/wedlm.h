@@ -1,0 +1,216 @@
+/*
+ * wedlm.h - C ABI of the WeDLM decoding-step library for NVIDIA B200 (sm_100a).
+ *
+ * One step of Streaming Parallel Decoding (Algorithm 1 of the WeDLM paper) works on a fixed
+ * window of W slots per sequence on top of a committed prefix whose keys/values live in a
+ * paged KV cache:
+ *
+ *   wedlm_reorder            Topological Reordering (Eq. 5-6): filled slots first, masks last,
+ *                            logical position ids kept; commit length of Algorithm 1.
+ *   wedlm_window_attn        RoPE at the logical ids (Section 2.2), staging of the window's
+ *                            K/V behind the prefix, causal attention of the reordered window
+ *                            over prefix + window (Section 5.2, "a small prefill"), GQA.
+ *   wedlm_kv_append          the staging step alone ("Extend (K, V)" of Algorithm 1).
+ *   wedlm_confidence_commit  per-mask-row entropy / max-prob / arg-max over the vocabulary,
+ *                            selection by distance-adjusted entropy (Eq. 11), then Commit,
+ *                            Predict and Refill of Algorithm 1.
+ *   wedlm_window_refill      Commit + shift + Refill alone.
+ *
+ * Conventions common to every call
+ *   - Every pointer named below is a DEVICE pointer unless it is the config or says "host".
+ *     The caller owns all memory; the library allocates and frees nothing and keeps no state
+ *     between calls.  Scratch memory is a caller-supplied workspace sized by a query function.
+ *   - Calls are asynchronous on the CUDA stream passed as `stream` (a cudaStream_t cast to
+ *     void*; NULL is the legacy default stream).  No call synchronises with the host.
+ *   - All tensors are dense, row-major ("last index fastest") and need 16-byte aligned base
+ *     addresses.  Index tensors are int32, flags are uint8.
+ *   - "logical order" = ascending position id within the window; "physical order" = the order
+ *     after wedlm_reorder.  Slot j (logical) of sequence b has position id prefix_len[b] + j.
+ *   - Return value: WEDLM_OK or a negative WEDLM_ERR_* code.  Argument errors are detected on
+ *     the host before anything is launched.  Data-dependent errors (a block-table entry outside
+ *     the page pool) are detected on the device: the offending access is skipped and a bit is
+ *     OR-ed into *status (if status != NULL); nothing traps.
+ */
+#ifndef WEDLM_H_
+#define WEDLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define WEDLM_OK                        0
+#define WEDLM_ERR_INVALID_ARG         (-1)
+#define WEDLM_ERR_UNSUPPORTED         (-2)
+#define WEDLM_ERR_WORKSPACE_TOO_SMALL (-3)
+#define WEDLM_ERR_CUDA                (-4)
+#define WEDLM_ERR_TIMEOUT             (-5)
+
+/* bits OR-ed into the device status word */
+#define WEDLM_STATUS_BAD_PAGE     1   /* block_table entry outside [0, num_pages)            */
+#define WEDLM_STATUS_BAD_LENGTH   2   /* prefix_len[b] < 0 or prefix_len[b]+W beyond the table */
+#define WEDLM_STATUS_WAIT_EXPIRED 4   /* a bounded on-chip wait gave up (tensor-core path)     */
+
+#define WEDLM_DTYPE_BF16 0
+#define WEDLM_DTYPE_F32  1
+
+#define WEDLM_CONF_ENTROPY 0   /* select mask i iff  H_i + lambda * d_i <= tau   (Eq. 11) */
+#define WEDLM_CONF_MAXPROB 1   /* select mask i iff  max_v p_i(v) >= maxprob_thr          */
+
+#define WEDLM_ATTN_AUTO    0
+#define WEDLM_ATTN_GENERIC 1   /* CUDA-core kernel, any supported shape, bf16 or fp32     */
+#define WEDLM_ATTN_TENSOR  2   /* tcgen05 + TMA kernel, bf16, head_dim 128, page 16       */
+
+typedef struct wedlm_config {
+  int32_t batch;              /* B  sequences                                              */
+  int32_t window;             /* W  slots per sequence (1..1024)                           */
+  int32_t n_q_heads;          /* Hq                                                        */
+  int32_t n_kv_heads;         /* Hkv, divides Hq; query head h reads KV head h / (Hq/Hkv)  */
+  int32_t head_dim;           /* D  (32, 64, 128 or 256)                                   */
+  int32_t page_size;          /* tokens per cache page (8, 16 or 32)                       */
+  int32_t max_pages_per_seq;  /* row stride of block_table                                 */
+  int32_t num_pages;          /* pages in the cache pool                                   */
+  int32_t vocab;              /* V                                                         */
+  int32_t dtype;              /* WEDLM_DTYPE_*: storage type of q/k/v/out, cache, logits   */
+  int32_t rope_style;         /* 0: pairs (d, d+D/2) "rotate-half"; 1: pairs (2d, 2d+1)    */
+  float   rope_theta;         /* angle of pair d at position p is p * theta^(-2d/D)        */
+  float   softmax_scale;      /* 0 selects 1/sqrt(D)                                       */
+  int32_t conf_mode;          /* WEDLM_CONF_*                                              */
+  float   tau;                /* entropy threshold (nats)                                  */
+  float   lambda;             /* distance penalty of Eq. 11                                */
+  float   maxprob_thr;
+  int32_t mask_token_id;      /* token id written into fresh mask slots                    */
+  int32_t max_prefix_len;     /* host-known upper bound of prefix_len[b]; sizes the grid   */
+  int32_t attn_impl;          /* WEDLM_ATTN_*                                              */
+} wedlm_config_t;
+
+/* Human-readable text of a return code.  Host pointer to a static string. */
+const char* wedlm_strerror(int code);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int wedlm_version(void);
+
+/* Measurement aids (no counterpart in the paper).
+ * wedlm_launch_count: kernels launched through this library by the calling process so far.
+ * wedlm_profile_next_attn: the next wedlm_window_attn call made by the calling host thread records
+ *   the two CUDA events (cudaEvent_t cast to void*, host handles, either may be NULL) on its stream
+ *   immediately before and after its main attention kernel, so that the kernel can be timed inside
+ *   a longer sequence of launches.  One-shot: the hook is cleared by that call. */
+unsigned long long wedlm_launch_count(void);
+int wedlm_profile_next_attn(void* event_before, void* event_after);
+
+/*
+ * Topological Reordering (Eq. 5-6) and commit length (Algorithm 1, Commit).
+ *   filled        in  u8  [B,W] logical order; non-zero = the slot holds a predicted token
+ *   window_tokens in  i32 [B,W] logical order, or NULL (then tokens_phys is not written)
+ *   prefix_len    in  i32 [B]
+ *   window_len    in  i32 [B] number of active slots (<= W), or NULL for W everywhere.
+ *                     Slots at or beyond window_len count as trailing masks.
+ *   perm          out i32 [B,W]  perm[i] = logical slot that sits at physical row i
+ *   inv_perm      out i32 [B,W]  inv_perm[perm[i]] = i
+ *   pos_ids       out i32 [B,W]  pos_ids[i] = prefix_len + perm[i]
+ *   tokens_phys   out i32 [B,W]  window_tokens[perm[i]], or NULL
+ *   n_filled      out i32 [B]    number of filled active slots (= first mask's physical row)
+ *   n_commit      out i32 [B]    length of the leading run of filled slots in logical order
+ */
+int wedlm_reorder(const wedlm_config_t* cfg, const uint8_t* filled, const int32_t* window_tokens,
+                  const int32_t* prefix_len, const int32_t* window_len,
+                  int32_t* perm, int32_t* inv_perm, int32_t* pos_ids, int32_t* tokens_phys,
+                  int32_t* n_filled, int32_t* n_commit, void* stream);
+
+/* Bytes of workspace wedlm_window_attn needs for this config (uses batch, window, heads,
+ * head_dim, dtype, max_prefix_len, attn_impl).  Returns 0 on an invalid config. */
+size_t wedlm_window_attn_workspace_bytes(const wedlm_config_t* cfg);
+
+/*
+ * One attention layer of the step's forward (Section 5.2; RoPE per Section 2.2).
+ *   q            in  [B,W,Hq,D]  window queries, physical order, before RoPE
+ *   k, v         in  [B,W,Hkv,D] window keys / values, physical order, k before RoPE
+ *   k_cache,
+ *   v_cache   in/out [num_pages,Hkv,page_size,D]  paged cache; K stored already rotated.
+ *                    Rows prefix_len[b] .. prefix_len[b]+W-1 of sequence b are OVERWRITTEN
+ *                    with the rotated k and v of physical rows 0..W-1 (staging).  Because the
+ *                    committed slots are the first physical rows, a later commit of n tokens
+ *                    is just prefix_len += n.  The pages covering prefix_len+W tokens must be
+ *                    present in the block table.
+ *   block_table  in  i32 [B,max_pages_per_seq]
+ *   prefix_len   in  i32 [B]
+ *   pos_ids      in  i32 [B,W]   from wedlm_reorder
+ *   out          out [B,W,Hq,D]  out[b,i,h] = softmax over {prefix} U {window rows j <= i} of
+ *                                scale * <q~, k~>, times V
+ *   kv_slot_idx  out i32 [B,W]   cache slot (page*page_size + offset) of physical row i, or NULL
+ *   workspace        scratch of at least wedlm_window_attn_workspace_bytes(cfg) bytes
+ *   status    in/out i32 [1] or NULL; WEDLM_STATUS_* bits are OR-ed in, never cleared
+ */
+int wedlm_window_attn(const wedlm_config_t* cfg, const void* q, const void* k, const void* v,
+                      void* k_cache, void* v_cache, const int32_t* block_table,
+                      const int32_t* prefix_len, const int32_t* pos_ids, void* out,
+                      int32_t* kv_slot_idx, void* workspace, size_t workspace_bytes,
+                      int32_t* status, void* stream);
+
+/*
+ * "Extend (K, V)" of Algorithm 1 as a call of its own: write rows i < count[b] of k, v to the
+ * cache positions prefix_len[b] + i of sequence b.
+ *   pos_ids   in i32 [B,W] or NULL.  Non-NULL: k is rotated at these positions before it is
+ *                stored.  NULL: k is stored as given (already rotated).
+ *   count     in i32 [B] or NULL (= W rows).
+ *   kv_slot_idx out i32 [B,W] or NULL; rows >= count are set to -1.
+ */
+int wedlm_kv_append(const wedlm_config_t* cfg, const void* k, const void* v, const int32_t* pos_ids,
+                    void* k_cache, void* v_cache, const int32_t* block_table,
+                    const int32_t* prefix_len, const int32_t* count, int32_t* kv_slot_idx,
+                    int32_t* status, void* stream);
+
+/* Bytes of workspace wedlm_confidence_commit needs (uses batch, window, vocab, dtype). */
+size_t wedlm_confidence_workspace_bytes(const wedlm_config_t* cfg);
+
+/*
+ * Confidence over the vocabulary (entropy of Section 5.2), selection by Eq. 11, and the Commit /
+ * Predict / Refill lines of Algorithm 1, for every sequence.
+ *   logits         in  [B,W,V]  physical order; only mask rows (n_filled[b] <= i < window_len[b])
+ *                               are read
+ *   perm, n_filled, n_commit  in   from wedlm_reorder of the same window state
+ *   window_tokens  in/out i32 [B,W] logical order
+ *   filled         in/out u8  [B,W]
+ *   prefix_len     in/out i32 [B]   += committed_count
+ *   window_len     in/out i32 [B] or NULL (= W, not written)
+ *   remaining_budget in/out i32 [B] or NULL (unlimited): fresh mask slots still allowed;
+ *                               Refill appends min(committed_count, budget)
+ *   argmax         out i32 [B,W] physical rows; -1 on rows that are not active masks
+ *   maxprob, entropy, lse  out f32 [B,W]; NaN on rows that are not active masks (each may be NULL)
+ *   committed_tokens out i32 [B,W] first committed_count[b] entries valid, rest -1
+ *   committed_count  out i32 [B]
+ *   filled_count     out i32 [B]  masks filled this step
+ * Order of operations per sequence: commit the n_commit leading slots; among the remaining
+ * masks compute d = logical distance to the leftmost mask; select; if nothing is selected and a
+ * mask exists, select the single best-scoring mask (leftmost on ties) so that decoding always
+ * progresses; write arg-max tokens into the selected slots; shift the window left by n_commit;
+ * append fresh masks.
+ */
+int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const int32_t* perm,
+                            const int32_t* n_filled, const int32_t* n_commit,
+                            int32_t* window_tokens, uint8_t* filled, int32_t* prefix_len,
+                            int32_t* window_len, int32_t* remaining_budget,
+                            int32_t* argmax, float* maxprob, float* entropy, float* lse,
+                            int32_t* committed_tokens, int32_t* committed_count,
+                            int32_t* filled_count, void* workspace, size_t workspace_bytes,
+                            void* stream);
+
+/*
+ * Commit + shift + Refill of Algorithm 1 alone, for callers that did the selection themselves
+ * and already wrote their fills into window_tokens / filled.
+ *   n_commit in i32 [B]  slots to commit (from wedlm_reorder, i.e. counted BEFORE the fills of
+ *                        this step: only those rows' K/V are cache-valid)
+ * Other arguments as in wedlm_confidence_commit.
+ */
+int wedlm_window_refill(const wedlm_config_t* cfg, const int32_t* n_commit,
+                        int32_t* window_tokens, uint8_t* filled, int32_t* prefix_len,
+                        int32_t* window_len, int32_t* remaining_budget,
+                        int32_t* committed_tokens, int32_t* committed_count, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WEDLM_H_ */

@@ -1,0 +1,213 @@
+// C ABI of the WeDLM step library: argument validation, workspace planning, kernel dispatch.
+#include <atomic>
+
+#include "common.cuh"
+
+using namespace wedlm;
+
+namespace {
+std::atomic<unsigned long long> g_launches{0};
+// One-shot profiling hook: events to record around the main attention kernel of the next
+// wedlm_window_attn call made by this thread.
+thread_local cudaEvent_t t_ev_before = nullptr;
+thread_local cudaEvent_t t_ev_after = nullptr;
+}  // namespace
+
+namespace wedlm {
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+}  // namespace wedlm
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Checks every field a call may rely on.  `need_vocab` / `need_cache` select the groups used.
+int check_config(const wedlm_config_t* c, bool need_cache, bool need_vocab) {
+  if (c == nullptr) return WEDLM_ERR_INVALID_ARG;
+  if (c->batch < 0 || c->window < 1 || c->window > 1024) return WEDLM_ERR_INVALID_ARG;
+  if (c->dtype != WEDLM_DTYPE_BF16 && c->dtype != WEDLM_DTYPE_F32) return WEDLM_ERR_INVALID_ARG;
+  if (need_cache) {
+    if (c->n_q_heads < 1 || c->n_kv_heads < 1 || c->n_q_heads % c->n_kv_heads != 0) return WEDLM_ERR_INVALID_ARG;
+    if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128 && c->head_dim != 256) return WEDLM_ERR_UNSUPPORTED;
+    if (c->page_size != 8 && c->page_size != 16 && c->page_size != 32) return WEDLM_ERR_UNSUPPORTED;
+    if (c->max_pages_per_seq < 1 || c->num_pages < 1) return WEDLM_ERR_INVALID_ARG;
+    if (c->rope_style != 0 && c->rope_style != 1) return WEDLM_ERR_INVALID_ARG;
+    if (!(c->rope_theta > 0.f) || c->softmax_scale < 0.f) return WEDLM_ERR_INVALID_ARG;
+    if (c->max_prefix_len < 0) return WEDLM_ERR_INVALID_ARG;
+    if ((long long)c->max_prefix_len + c->window > (long long)c->max_pages_per_seq * c->page_size) return WEDLM_ERR_INVALID_ARG;
+    if (c->attn_impl < WEDLM_ATTN_AUTO || c->attn_impl > WEDLM_ATTN_TENSOR) return WEDLM_ERR_INVALID_ARG;
+  }
+  if (need_vocab) {
+    if (c->vocab < 1) return WEDLM_ERR_INVALID_ARG;
+    if (c->conf_mode != WEDLM_CONF_ENTROPY && c->conf_mode != WEDLM_CONF_MAXPROB) return WEDLM_ERR_INVALID_ARG;
+    if (c->tau != c->tau || c->lambda != c->lambda || c->maxprob_thr != c->maxprob_thr) return WEDLM_ERR_INVALID_ARG;
+  }
+  return WEDLM_OK;
+}
+
+Shape make_shape(const wedlm_config_t* c) {
+  Shape s;
+  s.B = c->batch; s.W = c->window; s.Hq = c->n_q_heads; s.Hkv = c->n_kv_heads; s.D = c->head_dim;
+  s.G = c->n_kv_heads > 0 ? c->n_q_heads / c->n_kv_heads : 1;
+  s.page = c->page_size; s.max_pages = c->max_pages_per_seq; s.num_pages = c->num_pages; s.V = c->vocab;
+  s.dtype = c->dtype; s.rope_style = c->rope_style; s.theta = c->rope_theta;
+  s.scale = c->softmax_scale > 0.f ? c->softmax_scale : 1.0f / sqrtf((float)c->head_dim);
+  return s;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+namespace wedlm {
+
+AttnPlan plan_attention(const wedlm_config_t* c) {
+  AttnPlan p{};
+  const int elem = c->dtype == WEDLM_DTYPE_BF16 ? 2 : 4;
+  p.impl = WEDLM_ATTN_GENERIC;
+  const long long total = (long long)c->max_prefix_len + c->window;
+  const long long n_rb = (c->window + 15) / 16;
+  const long long units = (long long)c->batch * c->n_q_heads * n_rb;
+  long long want = units > 0 ? (148LL * 4 + units - 1) / units : 1;      // a few blocks per SM
+  long long cap = total / 256 > 1 ? total / 256 : 1;                      // keep chunks >= 256 keys
+  long long S = want < 1 ? 1 : (want > cap ? cap : want);
+  long long chunk = (total + S - 1) / S;
+  chunk = (chunk + c->page_size - 1) / c->page_size * c->page_size;
+  S = (total + chunk - 1) / chunk;
+  p.n_splits = (int)S;
+  p.chunk = (int)chunk;
+  p.q_rot_bytes = align_up((size_t)c->batch * c->window * c->n_q_heads * c->head_dim * elem, 256);
+  if (S > 1) {
+    size_t rows = (size_t)c->batch * c->n_q_heads * c->window * (size_t)S;
+    p.part_o_bytes = align_up(rows * c->head_dim * sizeof(float), 256);
+    p.part_ml_bytes = align_up(rows * 2 * sizeof(float), 256);
+  }
+  p.total_bytes = p.q_rot_bytes + p.part_o_bytes + p.part_ml_bytes;
+  return p;
+}
+
+}  // namespace wedlm
+
+extern "C" {
+
+const char* wedlm_strerror(int code) {
+  switch (code) {
+    case WEDLM_OK: return "ok";
+    case WEDLM_ERR_INVALID_ARG: return "invalid argument";
+    case WEDLM_ERR_UNSUPPORTED: return "unsupported configuration";
+    case WEDLM_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case WEDLM_ERR_CUDA: return "CUDA error";
+    case WEDLM_ERR_TIMEOUT: return "device wait expired";
+    default: return "unknown error code";
+  }
+}
+
+int wedlm_version(void) { return 100; }
+
+unsigned long long wedlm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int wedlm_profile_next_attn(void* event_before, void* event_after) {
+  t_ev_before = (cudaEvent_t)event_before;
+  t_ev_after = (cudaEvent_t)event_after;
+  return WEDLM_OK;
+}
+
+int wedlm_reorder(const wedlm_config_t* cfg, const uint8_t* filled, const int32_t* window_tokens,
+                  const int32_t* prefix_len, const int32_t* window_len, int32_t* perm, int32_t* inv_perm,
+                  int32_t* pos_ids, int32_t* tokens_phys, int32_t* n_filled, int32_t* n_commit, void* stream) {
+  int rc = check_config(cfg, false, false);
+  if (rc != WEDLM_OK) return rc;
+  if (cfg->batch == 0) return WEDLM_OK;
+  if (!filled || !prefix_len || !perm || !inv_perm || !pos_ids || !n_filled || !n_commit) return WEDLM_ERR_INVALID_ARG;
+  if (tokens_phys && !window_tokens) return WEDLM_ERR_INVALID_ARG;
+  return launch_reorder(make_shape(cfg), filled, window_tokens, prefix_len, window_len, perm, inv_perm, pos_ids,
+                        tokens_phys, n_filled, n_commit, (cudaStream_t)stream);
+}
+
+size_t wedlm_window_attn_workspace_bytes(const wedlm_config_t* cfg) {
+  if (check_config(cfg, true, false) != WEDLM_OK) return 0;
+  size_t b = plan_attention(cfg).total_bytes;
+  return b ? b : 256;
+}
+
+int wedlm_window_attn(const wedlm_config_t* cfg, const void* q, const void* k, const void* v, void* k_cache,
+                      void* v_cache, const int32_t* block_table, const int32_t* prefix_len, const int32_t* pos_ids,
+                      void* out, int32_t* kv_slot_idx, void* workspace, size_t workspace_bytes, int32_t* status,
+                      void* stream) {
+  int rc = check_config(cfg, true, false);
+  if (rc != WEDLM_OK) return rc;
+  if (cfg->batch == 0) return WEDLM_OK;
+  if (!q || !k || !v || !k_cache || !v_cache || !block_table || !prefix_len || !pos_ids || !out || !workspace)
+    return WEDLM_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(k_cache) || !aligned16(v_cache) ||
+      !aligned16(out) || !aligned16(workspace))
+    return WEDLM_ERR_INVALID_ARG;
+  AttnPlan plan = plan_attention(cfg);
+  if (workspace_bytes < plan.total_bytes) return WEDLM_ERR_WORKSPACE_TOO_SMALL;
+  Shape s = make_shape(cfg);
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = static_cast<char*>(workspace);
+  void* q_rot = ws;
+  float* part_o = reinterpret_cast<float*>(ws + plan.q_rot_bytes);
+  float* part_ml = reinterpret_cast<float*>(ws + plan.q_rot_bytes + plan.part_o_bytes);
+  rc = launch_rope_stage(s, q, k, v, q_rot, k_cache, v_cache, block_table, prefix_len, pos_ids, nullptr, kv_slot_idx,
+                         status, st);
+  if (rc != WEDLM_OK) return rc;
+  cudaEvent_t ev0 = t_ev_before, ev1 = t_ev_after;
+  t_ev_before = t_ev_after = nullptr;
+  if (ev0 && cudaEventRecord(ev0, st) != cudaSuccess) return WEDLM_ERR_CUDA;
+  rc = launch_attn_generic(s, plan, q_rot, k_cache, v_cache, block_table, prefix_len, out, part_o, part_ml, status, st);
+  if (ev1 && cudaEventRecord(ev1, st) != cudaSuccess) return WEDLM_ERR_CUDA;
+  if (rc != WEDLM_OK) return rc;
+  if (plan.n_splits > 1) rc = launch_attn_merge(s, plan, prefix_len, part_o, part_ml, out, st);
+  return rc;
+}
+
+int wedlm_kv_append(const wedlm_config_t* cfg, const void* k, const void* v, const int32_t* pos_ids, void* k_cache,
+                    void* v_cache, const int32_t* block_table, const int32_t* prefix_len, const int32_t* count,
+                    int32_t* kv_slot_idx, int32_t* status, void* stream) {
+  int rc = check_config(cfg, true, false);
+  if (rc != WEDLM_OK) return rc;
+  if (cfg->batch == 0) return WEDLM_OK;
+  if (!k || !v || !k_cache || !v_cache || !block_table || !prefix_len) return WEDLM_ERR_INVALID_ARG;
+  if (!aligned16(k) || !aligned16(v) || !aligned16(k_cache) || !aligned16(v_cache)) return WEDLM_ERR_INVALID_ARG;
+  return launch_rope_stage(make_shape(cfg), nullptr, k, v, nullptr, k_cache, v_cache, block_table, prefix_len, pos_ids,
+                           count, kv_slot_idx, status, (cudaStream_t)stream);
+}
+
+size_t wedlm_confidence_workspace_bytes(const wedlm_config_t* cfg) {
+  if (check_config(cfg, false, true) != WEDLM_OK) return 0;
+  size_t b = confidence_workspace_bytes(cfg);
+  return b ? b : 256;
+}
+
+int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const int32_t* perm,
+                            const int32_t* n_filled, const int32_t* n_commit, int32_t* window_tokens,
+                            uint8_t* filled, int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
+                            int32_t* argmax, float* maxprob, float* entropy, float* lse, int32_t* committed_tokens,
+                            int32_t* committed_count, int32_t* filled_count, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+  int rc = check_config(cfg, false, true);
+  if (rc != WEDLM_OK) return rc;
+  if (cfg->batch == 0) return WEDLM_OK;
+  if (!logits || !perm || !n_filled || !n_commit || !window_tokens || !filled || !prefix_len || !workspace)
+    return WEDLM_ERR_INVALID_ARG;
+  if (!aligned16(workspace)) return WEDLM_ERR_INVALID_ARG;
+  if (workspace_bytes < confidence_workspace_bytes(cfg)) return WEDLM_ERR_WORKSPACE_TOO_SMALL;
+  return launch_confidence(make_shape(cfg), cfg, logits, perm, n_filled, n_commit, window_tokens, filled, prefix_len,
+                           window_len, remaining_budget, argmax, maxprob, entropy, lse, committed_tokens,
+                           committed_count, filled_count, workspace, (cudaStream_t)stream);
+}
+
+int wedlm_window_refill(const wedlm_config_t* cfg, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
+                        int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
+                        int32_t* committed_tokens, int32_t* committed_count, void* stream) {
+  int rc = check_config(cfg, false, false);
+  if (rc != WEDLM_OK) return rc;
+  if (cfg->batch == 0) return WEDLM_OK;
+  if (!n_commit || !window_tokens || !filled || !prefix_len) return WEDLM_ERR_INVALID_ARG;
+  return launch_window_refill(make_shape(cfg), cfg, n_commit, window_tokens, filled, prefix_len, window_len,
+                              remaining_budget, committed_tokens, committed_count, (cudaStream_t)stream);
+}
+
+}  // extern "C"

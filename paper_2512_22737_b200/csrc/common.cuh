@@ -1,0 +1,88 @@
+// Shared device/host helpers of the WeDLM step library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "wedlm.h"
+
+namespace wedlm {
+
+// Launch descriptors handed from the C-ABI layer to the kernels' host launchers.
+struct Shape {
+  int B, W, Hq, Hkv, D, G;
+  int page, max_pages, num_pages, V;
+  int dtype, rope_style;
+  float theta, scale;
+};
+
+__device__ __forceinline__ float ld_as_float(const float* p, size_t i) { return p[i]; }
+__device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p, size_t i) { return __bfloat162float(p[i]); }
+__device__ __forceinline__ void st_from_float(float* p, size_t i, float x) { p[i] = x; }
+__device__ __forceinline__ void st_from_float(__nv_bfloat16* p, size_t i, float x) { p[i] = __float2bfloat16_rn(x); }
+
+// Physical cache row (page * page_size + offset) of token position t of sequence b, or -1 with a
+// status bit when the block table points outside the pool.
+__device__ __forceinline__ long long cache_slot(const int32_t* __restrict__ block_table, int b, int t,
+                                                int page, int max_pages, int num_pages, int32_t* status) {
+  int lp = t / page;
+  if (t < 0 || lp >= max_pages) {
+    if (status) atomicOr(status, WEDLM_STATUS_BAD_LENGTH);
+    return -1;
+  }
+  int pp = block_table[(size_t)b * max_pages + lp];
+  if (pp < 0 || pp >= num_pages) {
+    if (status) atomicOr(status, WEDLM_STATUS_BAD_PAGE);
+    return -1;
+  }
+  return (long long)pp * page + (t - lp * page);
+}
+
+// Element offset of (slot, kv head g, dim 0) in a cache laid out [num_pages][Hkv][page][D].
+__device__ __forceinline__ size_t cache_offset(long long slot, int g, int page, int Hkv, int D) {
+  long long pp = slot / page;
+  int off = (int)(slot - pp * page);
+  return (((size_t)pp * Hkv + g) * page + off) * (size_t)D;
+}
+
+// Host launchers (defined in the .cu files).
+int launch_reorder(const Shape& s, const uint8_t* filled, const int32_t* window_tokens, const int32_t* prefix_len,
+                   const int32_t* window_len, int32_t* perm, int32_t* inv_perm, int32_t* pos_ids,
+                   int32_t* tokens_phys, int32_t* n_filled, int32_t* n_commit, cudaStream_t st);
+
+int launch_rope_stage(const Shape& s, const void* q, const void* k, const void* v, void* q_rot, void* k_cache,
+                      void* v_cache, const int32_t* block_table, const int32_t* prefix_len, const int32_t* pos_ids,
+                      const int32_t* count, int32_t* kv_slot_idx, int32_t* status, cudaStream_t st);
+
+struct AttnPlan {
+  int impl;            // WEDLM_ATTN_GENERIC or WEDLM_ATTN_TENSOR
+  int n_splits;        // key chunks per (sequence, head)
+  int chunk;           // keys per chunk (multiple of the page size)
+  size_t q_rot_bytes, part_o_bytes, part_ml_bytes, total_bytes;
+};
+AttnPlan plan_attention(const wedlm_config_t* cfg);
+
+int launch_attn_generic(const Shape& s, const AttnPlan& plan, const void* q_rot, const void* k_cache,
+                        const void* v_cache, const int32_t* block_table, const int32_t* prefix_len, void* out,
+                        float* part_o, float* part_ml, int32_t* status, cudaStream_t st);
+
+int launch_attn_merge(const Shape& s, const AttnPlan& plan, const int32_t* prefix_len, const float* part_o,
+                      const float* part_ml, void* out, cudaStream_t st);
+
+size_t confidence_workspace_bytes(const wedlm_config_t* cfg);
+int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* logits, const int32_t* perm,
+                      const int32_t* n_filled, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
+                      int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget, int32_t* argmax,
+                      float* maxprob, float* entropy, float* lse, int32_t* committed_tokens,
+                      int32_t* committed_count, int32_t* filled_count, void* workspace, cudaStream_t st);
+
+int launch_window_refill(const Shape& s, const wedlm_config_t* cfg, const int32_t* n_commit, int32_t* window_tokens,
+                         uint8_t* filled, int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
+                         int32_t* committed_tokens, int32_t* committed_count, cudaStream_t st);
+
+inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? WEDLM_OK : WEDLM_ERR_CUDA; }
+
+// Number of kernels this process has launched through the library (reported by wedlm_launch_count).
+void count_launch(int n = 1);
+
+}  // namespace wedlm

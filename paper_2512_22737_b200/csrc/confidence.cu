@@ -1,0 +1,348 @@
+// Per-mask-row confidence over the vocabulary (entropy of Section 5.2; max-prob), selection by the
+// distance-adjusted entropy of Eq. 11, and the Commit / Predict / Refill lines of Algorithm 1.
+//
+// Pass 1 (conf_partial_kernel) streams the logits of the mask rows once with 16-byte loads and
+// reduces each chunk of a row to (m, s, t, a):  m = max x, a = lowest index attaining it,
+// s = sum e^(x-m), t = sum (x-m) e^(x-m).  Pass 2 (conf_commit_kernel, one warp per sequence)
+// merges the chunks of every row in double precision, lse = m + ln s, p_max = 1/s,
+// H = ln s - t/s, then runs the window update.
+#include <math_constants.h>
+
+#include "common.cuh"
+
+namespace wedlm {
+
+constexpr int kConfThreads = 256;
+constexpr int kConfVecs = 4;    // 16-byte loads in flight per thread
+
+template <typename T> struct VecTraits;
+template <> struct VecTraits<__nv_bfloat16> { static constexpr int VL = 8; };
+template <> struct VecTraits<float> { static constexpr int VL = 4; };
+
+template <typename T>
+__host__ __device__ constexpr int conf_chunk_elems() { return kConfThreads * kConfVecs * VecTraits<T>::VL; }
+
+__device__ __forceinline__ void unpack16(const uint4& u, float (&x)[8]) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    x[2 * e] = __uint_as_float(w[e] << 16);
+    x[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ void unpack16(const uint4& u, float (&x)[4]) {
+  x[0] = __uint_as_float(u.x); x[1] = __uint_as_float(u.y); x[2] = __uint_as_float(u.z); x[3] = __uint_as_float(u.w);
+}
+
+// (value, index) arg-max combine: larger value wins, equal values keep the lower index.
+__device__ __forceinline__ void argmax_combine(float& v, int& i, float ov, int oi) {
+  if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+}
+
+// 1-D grid over (row, chunk) with the chunk index fastest; rows that are not active masks exit.
+template <typename T, bool VEC>
+__global__ void __launch_bounds__(kConfThreads)
+conf_partial_kernel(int W, int V, int n_chunks, const T* __restrict__ logits, const int32_t* __restrict__ n_filled,
+                    const int32_t* __restrict__ window_len, float4* __restrict__ part) {
+  constexpr int VL = VecTraits<T>::VL;
+  constexpr int EPT = kConfVecs * VL;
+  constexpr int CHUNK = conf_chunk_elems<T>();
+  const int row = blockIdx.x / n_chunks, chunk = blockIdx.x - row * n_chunks;
+  const int b = row / W, i = row - b * W;
+  const int L = window_len ? min(max(window_len[b], 0), W) : W;
+  if (i < n_filled[b] || i >= L) return;
+  const int tid = threadIdx.x;
+  const int base = chunk * CHUNK;
+  const T* src = logits + (size_t)row * V;
+
+  float x[EPT];
+  if (VEC) {
+    uint4 raw[kConfVecs];
+#pragma unroll
+    for (int k = 0; k < kConfVecs; ++k) {
+      int e0 = base + (k * kConfThreads + tid) * VL;
+      if (e0 < V) raw[k] = __ldcs(reinterpret_cast<const uint4*>(src + e0));   // V % VL == 0 on this path
+    }
+#pragma unroll
+    for (int k = 0; k < kConfVecs; ++k) {
+      int e0 = base + (k * kConfThreads + tid) * VL;
+      float xv[VL];
+      if (e0 < V) unpack16(raw[k], xv);
+#pragma unroll
+      for (int e = 0; e < VL; ++e) x[k * VL + e] = (e0 < V) ? xv[e] : -CUDART_INF_F;
+    }
+  } else {
+#pragma unroll
+    for (int k = 0; k < kConfVecs; ++k)
+#pragma unroll
+      for (int e = 0; e < VL; ++e) {
+        int idx = base + (k * kConfThreads + tid) * VL + e;
+        x[k * VL + e] = idx < V ? ld_as_float(src, idx) : -CUDART_INF_F;
+      }
+  }
+  // thread-local arg-max in increasing index order (strict > keeps the lowest index)
+  float m = -CUDART_INF_F;
+  int a = 0x7fffffff;
+#pragma unroll
+  for (int k = 0; k < kConfVecs; ++k)
+#pragma unroll
+    for (int e = 0; e < VL; ++e) {
+      int idx = base + (k * kConfThreads + tid) * VL + e;
+      if (x[k * VL + e] > m) { m = x[k * VL + e]; a = idx; }
+    }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    float ov = __shfl_xor_sync(0xffffffffu, m, o);
+    int oi = __shfl_xor_sync(0xffffffffu, a, o);
+    argmax_combine(m, a, ov, oi);
+  }
+  __shared__ float sm_m[kConfThreads / 32];
+  __shared__ int sm_a[kConfThreads / 32];
+  __shared__ float sm_s[kConfThreads / 32];
+  __shared__ float sm_t[kConfThreads / 32];
+  const int warp = tid >> 5, lane = tid & 31;
+  if (lane == 0) { sm_m[warp] = m; sm_a[warp] = a; }
+  __syncthreads();
+  m = sm_m[0]; a = sm_a[0];
+#pragma unroll
+  for (int w = 1; w < kConfThreads / 32; ++w) argmax_combine(m, a, sm_m[w], sm_a[w]);
+
+  // sums relative to the chunk maximum; terms whose exponential underflows to 0 add 0
+  float s = 0.f, t = 0.f;
+  if (m > -CUDART_INF_F) {
+#pragma unroll
+    for (int k = 0; k < EPT; ++k) {
+      float d = x[k] - m;
+      float e = exp2f(d * 1.4426950408889634f);
+      s += e;
+      t += (e > 0.f) ? d * e : 0.f;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, o);
+    t += __shfl_xor_sync(0xffffffffu, t, o);
+  }
+  if (lane == 0) { sm_s[warp] = s; sm_t[warp] = t; }
+  __syncthreads();
+  if (tid == 0) {
+    float ss = 0.f, tt = 0.f;
+#pragma unroll
+    for (int w = 0; w < kConfThreads / 32; ++w) { ss += sm_s[w]; tt += sm_t[w]; }
+    part[(size_t)row * n_chunks + chunk] = make_float4(m, ss, tt, __int_as_float(a));
+  }
+}
+
+// Commit + shift + Refill of Algorithm 1 for one sequence, executed by one warp.  tok_s / fil_s hold
+// the window in logical order with this step's fills already applied.
+__device__ void commit_shift_refill(int b, int W, int L, int n, const int* tok_s, const uint8_t* fil_s,
+                                    int mask_id, int32_t* window_tokens, uint8_t* filled, int32_t* prefix_len,
+                                    int32_t* window_len, int32_t* remaining_budget, int32_t* committed_tokens,
+                                    int32_t* committed_count) {
+  const int lane = threadIdx.x & 31;
+  const size_t o = (size_t)b * W;
+  n = min(max(n, 0), L);
+  int r = n;
+  if (remaining_budget) r = min(n, max(remaining_budget[b], 0));
+  const int new_len = L - n + r;
+  for (int j = lane; j < W; j += 32) {
+    if (committed_tokens) committed_tokens[o + j] = j < n ? tok_s[j] : -1;
+    int src = j + n;
+    bool keep = j < L - n;          // slot shifted down from position j + n
+    window_tokens[o + j] = keep ? tok_s[src] : mask_id;
+    filled[o + j] = keep ? fil_s[src] : (uint8_t)0;
+  }
+  if (lane == 0) {
+    if (committed_count) committed_count[b] = n;
+    prefix_len[b] += n;
+    if (window_len) window_len[b] = new_len;
+    if (remaining_budget) remaining_budget[b] = max(remaining_budget[b], 0) - r;
+  }
+}
+
+struct ConfParams {
+  int W, n_chunks, conf_mode, mask_id;
+  float tau, lambda, thr;
+};
+
+// One warp per sequence.
+__global__ void __launch_bounds__(32)
+conf_commit_kernel(ConfParams p, const float4* __restrict__ part, const int32_t* __restrict__ perm,
+                   const int32_t* __restrict__ n_filled, const int32_t* __restrict__ n_commit,
+                   int32_t* window_tokens, uint8_t* filled, int32_t* prefix_len, int32_t* window_len,
+                   int32_t* remaining_budget, int32_t* argmax, float* maxprob, float* entropy, float* lse,
+                   int32_t* committed_tokens, int32_t* committed_count, int32_t* filled_count) {
+  extern __shared__ unsigned char sm_raw[];
+  const int W = p.W;
+  double* score = reinterpret_cast<double*>(sm_raw);        // [W] per mask k
+  int* am = reinterpret_cast<int*>(score + W);                // [W] arg-max per mask k
+  int* tok_s = am + W;                                        // [W] logical
+  uint8_t* fil_s = reinterpret_cast<uint8_t*>(tok_s + W);     // [W] logical
+  uint8_t* pass = fil_s + W;                                  // [W] per mask k
+
+  const int b = blockIdx.x, lane = threadIdx.x;
+  const size_t o = (size_t)b * W;
+  const int L = window_len ? min(max(window_len[b], 0), W) : W;
+  const int nf = min(max(n_filled[b], 0), L);
+  const int n_mask = L - nf;
+  const float qnan = __int_as_float(0x7fc00000);
+
+  for (int j = lane; j < W; j += 32) {
+    tok_s[j] = window_tokens[o + j];
+    fil_s[j] = (j < L && filled[o + j]) ? 1 : 0;
+  }
+  // rows that are not active masks carry no statistics
+  for (int i = lane; i < W; i += 32) {
+    if (i < nf || i >= L) {
+      if (argmax) argmax[o + i] = -1;
+      if (maxprob) maxprob[o + i] = qnan;
+      if (entropy) entropy[o + i] = qnan;
+      if (lse) lse[o + i] = qnan;
+    }
+  }
+  const int j0 = n_mask > 0 ? perm[o + nf] : 0;
+  int n_pass = 0;
+  for (int k = lane; k < n_mask; k += 32) {
+    const int i = nf + k;
+    const float4* pr = part + (o + i) * p.n_chunks;
+    float m = -CUDART_INF_F;
+    int a = 0x7fffffff;
+    for (int c = 0; c < p.n_chunks; ++c) {
+      float4 v = pr[c];
+      argmax_combine(m, a, v.x, __float_as_int(v.w));     // chunks ascend in index, ties keep the lower
+    }
+    double s = 0.0, t = 0.0;
+    for (int c = 0; c < p.n_chunks; ++c) {
+      float4 v = pr[c];
+      if (v.x > -CUDART_INF_F) {
+        double dm = (double)v.x - (double)m;
+        double w = exp(dm);
+        s += w * (double)v.y;
+        t += w * ((double)v.z + dm * (double)v.y);
+      }
+    }
+    const double ln_s = log(s);
+    const double H = ln_s - t / s;
+    const double pmax = 1.0 / s;
+    if (argmax) argmax[o + i] = a;
+    if (maxprob) maxprob[o + i] = (float)pmax;
+    if (entropy) entropy[o + i] = (float)H;
+    if (lse) lse[o + i] = (float)((double)m + ln_s);
+    const int j = perm[o + i];
+    double sc;
+    bool ok;
+    if (p.conf_mode == WEDLM_CONF_ENTROPY) {
+      sc = H + (double)p.lambda * (double)(j - j0);           // Eq. 11
+      ok = sc <= (double)p.tau;
+    } else {
+      sc = -pmax;
+      ok = pmax >= (double)p.thr;
+    }
+    score[k] = sc;
+    am[k] = a;
+    pass[k] = ok ? 1 : 0;
+    n_pass += ok ? 1 : 0;
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) n_pass += __shfl_xor_sync(0xffffffffu, n_pass, off);
+  __syncwarp();
+  if (n_pass == 0 && n_mask > 0) {
+    // nothing passed: fill the single best-scoring mask, leftmost on ties
+    double best = CUDART_INF;
+    int bk = 0x7fffffff;
+    for (int k = lane; k < n_mask; k += 32)
+      if (score[k] < best || (score[k] == best && k < bk)) { best = score[k]; bk = k; }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      double ob = __shfl_xor_sync(0xffffffffu, best, off);
+      int ok_ = __shfl_xor_sync(0xffffffffu, bk, off);
+      if (ob < best || (ob == best && ok_ < bk)) { best = ob; bk = ok_; }
+    }
+    if (bk == 0x7fffffff) bk = 0;     // every score NaN: still make progress at the leftmost mask
+    if (lane == 0) pass[bk] = 1;
+    n_pass = 1;
+  }
+  __syncwarp();
+  for (int k = lane; k < n_mask; k += 32) {
+    if (pass[k]) {
+      const int j = perm[o + nf + k];
+      tok_s[j] = am[k];
+      fil_s[j] = 1;
+    }
+  }
+  if (lane == 0 && filled_count) filled_count[b] = n_pass;
+  __syncwarp();
+  commit_shift_refill(b, W, L, n_commit[b], tok_s, fil_s, p.mask_id, window_tokens, filled, prefix_len, window_len,
+                      remaining_budget, committed_tokens, committed_count);
+}
+
+__global__ void __launch_bounds__(32)
+window_refill_kernel(int W, int mask_id, const int32_t* __restrict__ n_commit, int32_t* window_tokens,
+                     uint8_t* filled, int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
+                     int32_t* committed_tokens, int32_t* committed_count) {
+  extern __shared__ unsigned char sm_raw[];
+  int* tok_s = reinterpret_cast<int*>(sm_raw);
+  uint8_t* fil_s = reinterpret_cast<uint8_t*>(tok_s + W);
+  const int b = blockIdx.x, lane = threadIdx.x;
+  const size_t o = (size_t)b * W;
+  const int L = window_len ? min(max(window_len[b], 0), W) : W;
+  for (int j = lane; j < W; j += 32) {
+    tok_s[j] = window_tokens[o + j];
+    fil_s[j] = (j < L && filled[o + j]) ? 1 : 0;
+  }
+  __syncwarp();
+  commit_shift_refill(b, W, L, n_commit[b], tok_s, fil_s, mask_id, window_tokens, filled, prefix_len, window_len,
+                      remaining_budget, committed_tokens, committed_count);
+}
+
+static int conf_chunks(const wedlm_config_t* cfg) {
+  int ce = cfg->dtype == WEDLM_DTYPE_BF16 ? conf_chunk_elems<__nv_bfloat16>() : conf_chunk_elems<float>();
+  return (cfg->vocab + ce - 1) / ce;
+}
+
+size_t confidence_workspace_bytes(const wedlm_config_t* cfg) {
+  return (size_t)cfg->batch * cfg->window * conf_chunks(cfg) * sizeof(float4);
+}
+
+int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* logits, const int32_t* perm,
+                      const int32_t* n_filled, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
+                      int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget, int32_t* argmax,
+                      float* maxprob, float* entropy, float* lse, int32_t* committed_tokens,
+                      int32_t* committed_count, int32_t* filled_count, void* workspace, cudaStream_t st) {
+  const int n_chunks = conf_chunks(cfg);
+  const long long blocks = (long long)s.B * s.W * n_chunks;
+  if (blocks > 0x7fffffffLL) return WEDLM_ERR_UNSUPPORTED;
+  float4* part = reinterpret_cast<float4*>(workspace);
+  if (s.dtype == WEDLM_DTYPE_BF16) {
+    using T = __nv_bfloat16;
+    const bool vec = (s.V % VecTraits<T>::VL == 0) && ((uintptr_t)logits % 16 == 0);
+    if (vec) conf_partial_kernel<T, true><<<(unsigned)blocks, kConfThreads, 0, st>>>(s.W, s.V, n_chunks, (const T*)logits, n_filled, window_len, part);
+    else     conf_partial_kernel<T, false><<<(unsigned)blocks, kConfThreads, 0, st>>>(s.W, s.V, n_chunks, (const T*)logits, n_filled, window_len, part);
+  } else {
+    using T = float;
+    const bool vec = (s.V % VecTraits<T>::VL == 0) && ((uintptr_t)logits % 16 == 0);
+    if (vec) conf_partial_kernel<T, true><<<(unsigned)blocks, kConfThreads, 0, st>>>(s.W, s.V, n_chunks, (const T*)logits, n_filled, window_len, part);
+    else     conf_partial_kernel<T, false><<<(unsigned)blocks, kConfThreads, 0, st>>>(s.W, s.V, n_chunks, (const T*)logits, n_filled, window_len, part);
+  }
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return WEDLM_ERR_CUDA;
+  ConfParams p{s.W, n_chunks, cfg->conf_mode, cfg->mask_token_id, cfg->tau, cfg->lambda, cfg->maxprob_thr};
+  size_t smem = (size_t)s.W * (sizeof(double) + 2 * sizeof(int) + 2);
+  conf_commit_kernel<<<s.B, 32, smem, st>>>(p, part, perm, n_filled, n_commit, window_tokens, filled, prefix_len,
+                                            window_len, remaining_budget, argmax, maxprob, entropy, lse,
+                                            committed_tokens, committed_count, filled_count);
+  count_launch();
+  return cuda_ok(cudaGetLastError());
+}
+
+int launch_window_refill(const Shape& s, const wedlm_config_t* cfg, const int32_t* n_commit, int32_t* window_tokens,
+                         uint8_t* filled, int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
+                         int32_t* committed_tokens, int32_t* committed_count, cudaStream_t st) {
+  size_t smem = (size_t)s.W * (sizeof(int) + 1);
+  window_refill_kernel<<<s.B, 32, smem, st>>>(s.W, cfg->mask_token_id, n_commit, window_tokens, filled, prefix_len,
+                                              window_len, remaining_budget, committed_tokens, committed_count);
+  count_launch();
+  return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace wedlm

@@ -1,0 +1,226 @@
+"""GPU-vs-oracle parity of the whole step, through the C-ABI binding.
+
+Small cases are compared element by element; the full-size serving and long-context workloads
+are compared on every integer output and on sampled attention vectors / confidence rows the
+oracle can compute one at a time."""
+import numpy as np
+import pytest
+import torch
+
+from workloads import get_config, make_step
+from oracle import wedlm_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = ["generic"]
+
+
+def _small_qwen(**kw):
+    base = get_config("cfg2_qwen_b1").replace(vocab=20000)
+    return base.replace(**kw)
+
+
+@pytest.mark.parametrize("seed", [251222737, 1, 2])
+def test_cfg1_tiny_fp32(seed):
+    import parity_util as pu
+    cfg = get_config("cfg1_tiny")
+    r = pu.full_parity(cfg, make_step(cfg, seed=seed))
+    assert r["attn_err"] < 1e-4          # fp32 end to end
+
+
+def test_cfg1_tiny_with_boost_exercises_the_threshold_branch():
+    import parity_util as pu
+    cfg = get_config("cfg1_tiny").replace(boost=12.0, boost_prob=0.6)
+    for seed in (3, 4, 5):
+        r = pu.full_parity(cfg, make_step(cfg, seed=seed))
+        assert r["attn_err"] < 1e-4
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_cfg2_qwen_single_sequence(impl):
+    import parity_util as pu
+    cfg = get_config("cfg2_qwen_b1")
+    r = pu.full_parity(cfg, make_step(cfg), attn_impl=impl)
+    print("cfg2 attention error", r["attn_err"], "excluded", r["excluded"])
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("boost", [14.4, 16.4, 20.4])
+def test_cfg2_calibrated_boosts_mixed_decisions(impl, boost):
+    """Boosts near 12.4 + s put rows on either side of tau = 0.3 (the literal +8 never passes)."""
+    import parity_util as pu
+    cfg = get_config("cfg2_qwen_b1").replace(boost=boost, boost_prob=0.7)
+    r = pu.full_parity(cfg, make_step(cfg, seed=11), attn_impl=impl)
+    assert r["excluded"] <= 1
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("B,W,lo,hi", [(3, 16, 0, 40), (4, 32, 100, 700), (2, 64, 1000, 1100), (5, 5, 1, 300), (2, 1, 17, 17)])
+def test_ragged_batches_span_tiles_and_tails(impl, B, W, lo, hi):
+    import parity_util as pu
+    cfg = _small_qwen(batch=B, window=W, prefix_lo=lo, prefix_hi=hi, obs_prob_lo=0.1, obs_prob_hi=0.7,
+                      boost=12.0, boost_prob=0.5, name="ragged")
+    pu.full_parity(cfg, make_step(cfg, seed=B * 100 + W), attn_impl=impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("Hq,Hkv,D", [(4, 4, 64), (8, 1, 128), (2, 1, 32), (6, 2, 256)])
+def test_head_geometries(impl, Hq, Hkv, D):
+    import parity_util as pu
+    cfg = _small_qwen(batch=2, window=8, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, prefix_lo=5, prefix_hi=90,
+                      vocab=3000, name="heads")
+    pu.full_parity(cfg, make_step(cfg, seed=Hq * 7 + D), attn_impl="generic")
+
+
+@pytest.mark.parametrize("P", [0, 1, 15, 16, 17, 31, 33])
+def test_page_boundaries(P):
+    import parity_util as pu
+    cfg = _small_qwen(batch=1, window=24, prefix_lo=P, prefix_hi=P, vocab=1000, name="pages")
+    pu.full_parity(cfg, make_step(cfg, seed=P), attn_impl="generic")
+
+
+def test_degenerate_windows():
+    import parity_util as pu
+    cfg = _small_qwen(batch=3, window=16, prefix_lo=30, prefix_hi=60, vocab=5000, name="degenerate")
+    inp = make_step(cfg, seed=9)
+    for pattern in (np.ones((3, 16), np.uint8), np.zeros((3, 16), np.uint8)):
+        inp2 = make_step(cfg, seed=9, filled=pattern)
+        pu.full_parity(cfg, inp2)
+    # leading run then a gap
+    f = np.zeros((3, 16), np.uint8)
+    f[:, :5] = 1
+    f[:, 7:9] = 1
+    pu.full_parity(cfg, make_step(cfg, seed=9, filled=f))
+
+
+def test_short_windows_and_budget():
+    import parity_util as pu
+    cfg = _small_qwen(batch=4, window=8, prefix_lo=10, prefix_hi=50, vocab=2000, boost=14.0, boost_prob=0.8,
+                      name="short")
+    f = np.array([[1, 1, 0, 1, 0, 0, 1, 1], [1, 1, 1, 1, 1, 0, 0, 0], [0, 1, 1, 0, 0, 0, 0, 0], [1, 1, 1, 0, 0, 0, 0, 0]], np.uint8)
+    inp = make_step(cfg, seed=21, filled=f)
+    pu.full_parity(cfg, inp, window_len=[8, 5, 3, 3], remaining_budget=[100, 2, 0, 1])
+
+
+def test_maxprob_mode_bf16():
+    import parity_util as pu
+    cfg = _small_qwen(batch=2, window=16, prefix_lo=40, prefix_hi=80, vocab=4096, conf_mode="maxprob",
+                      maxprob_thr=0.9, boost=13.0, boost_prob=0.6, name="maxprob")
+    pu.full_parity(cfg, make_step(cfg, seed=31))
+
+
+def test_unaligned_vocab_takes_the_scalar_path():
+    import parity_util as pu
+    cfg = _small_qwen(batch=2, window=8, prefix_lo=20, prefix_hi=20, vocab=10007, boost=11.0, name="oddvocab")
+    pu.full_parity(cfg, make_step(cfg, seed=41))
+
+
+def test_empty_batch_is_a_noop():
+    import paper_2512_22737_b200 as w
+    cfg = w.make_config(batch=0, window=8, n_q_heads=4, n_kv_heads=2, head_dim=64, max_pages_per_seq=4,
+                        num_pages=4, vocab=100)
+    e = torch.empty(0, dtype=torch.int32, device="cuda")
+    w.wedlm_reorder(cfg, torch.empty(0, dtype=torch.uint8, device="cuda"), None, e, None, e, e, e, None, e, e)
+    torch.cuda.synchronize()
+
+
+def test_bad_block_table_sets_status_and_does_not_fault():
+    import paper_2512_22737_b200 as w
+    import parity_util as pu
+    cfg = _small_qwen(batch=2, window=8, prefix_lo=40, prefix_hi=40, vocab=1000, name="badpage")
+    inp = make_step(cfg, seed=5)
+    inp["block_table"][1, 1] = inp["k_cache"].shape[0] + 7        # outside the pool
+    step, d = pu.run_gpu_step(cfg, inp)
+    assert int(step.status.item()) & w.binding.WEDLM_STATUS_BAD_PAGE
+    assert torch.isfinite(step.out.float()).all()
+    # the untouched sequence is still right
+    inp_ok = make_step(cfg, seed=5)
+    ref = pu.oracle_step(cfg, inp_ok)
+    err = pu.attn_vector_error(pu.bf16_from_device(step.out)[0], ref["out"][0])
+    assert err.max() <= pu.ATTN_REL_TOL
+
+
+def test_kv_append_alone_and_window_refill_alone():
+    import paper_2512_22737_b200 as w
+    import parity_util as pu
+    cfg = _small_qwen(batch=3, window=8, prefix_lo=10, prefix_hi=70, vocab=1000, name="append")
+    inp = make_step(cfg, seed=6)
+    d = pu.device_inputs(inp)
+    c = w.config_for(cfg, max_pages_per_seq=inp["block_table"].shape[1], num_pages=inp["k_cache"].shape[0],
+                     max_prefix_len=int(inp["prefix_len"].max()))
+    ro = orc.reorder(inp["filled"], inp["prefix_len"])
+    pos = torch.tensor(ro["pos_ids"], dtype=torch.int32, device="cuda")
+    count = torch.tensor([8, 3, 0], dtype=torch.int32, device="cuda")
+    slots = torch.empty(3, 8, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    k_before = d["k_cache"].clone()
+    w.wedlm_kv_append(c, d["k"], d["v"], pos, d["k_cache"], d["v_cache"], d["block_table"], d["prefix_len"], count,
+                      slots, status)
+    torch.cuda.synchronize()
+    want_slots = orc.stage_slots(inp["block_table"], inp["prefix_len"], 8, cfg.page_size)
+    want_slots[1, 3:] = -1
+    want_slots[2, :] = -1
+    np.testing.assert_array_equal(slots.cpu().numpy(), want_slots)
+    k_rot = orc.rope(orc.to_f64(inp["k"]), ro["pos_ids"][:, :, None], cfg.rope_theta)
+    kc = pu.bf16_from_device(d["k_cache"])
+    changed = (d["k_cache"] != k_before).any(dim=(1, 3)).sum().item()
+    assert changed <= 11 * cfg.n_kv_heads
+    for b, n in ((0, 8), (1, 3)):
+        for i in range(n):
+            s = int(want_slots[b, i])
+            got = kc[s // 16, :, s % 16]
+            want = orc.round_to_bf16(k_rot[b, i])
+            assert (np.abs(got - want) <= np.abs(want) * 2.0 ** -7 + 1e-30).all()
+    # refill alone
+    n_commit = torch.tensor(ro["n_commit"], dtype=torch.int32, device="cuda")
+    ct = torch.empty(3, 8, dtype=torch.int32, device="cuda")
+    cc = torch.empty(3, dtype=torch.int32, device="cuda")
+    w.wedlm_window_refill(c, n_commit, d["window_tokens"], d["filled"], d["prefix_len"], None, None, ct, cc)
+    torch.cuda.synchronize()
+    for b in range(3):
+        n = int(ro["n_commit"][b])
+        assert cc[b].item() == n
+        assert ct[b, :n].cpu().tolist() == inp["window_tokens"][b, :n].tolist()
+        want_tok = inp["window_tokens"][b, n:].tolist() + [cfg.mask_token_id] * n
+        want_fil = inp["filled"][b, n:].tolist() + [0] * n
+        assert d["window_tokens"][b].cpu().tolist() == want_tok
+        assert d["filled"][b].cpu().tolist() == want_fil
+        assert d["prefix_len"][b].item() == inp["prefix_len"][b] + n
+
+
+def _sampled_full_size(cfg_name, impl, n_attn=24, n_rows=24):
+    import parity_util as pu
+    cfg = get_config(cfg_name)
+    inp = make_step(cfg)
+    step, d = pu.run_gpu_step(cfg, inp, attn_impl=impl)
+    ref = pu.oracle_step(cfg, inp, with_attention=False)        # integers + confidence on every mask row
+    pu.check_reorder(step, ref)
+    np.testing.assert_array_equal(step.kv_slot_idx.cpu().numpy(), ref["kv_slot_idx"])
+    assert int(step.status.item()) == 0
+    excluded = pu.check_confidence_and_commit(cfg, step, d, inp, ref)
+    got = pu.bf16_from_device(step.out)
+    assert np.isfinite(got).all()
+    rng = np.random.default_rng(0)
+    B, W, Hq = cfg.batch, cfg.window, cfg.n_q_heads
+    worst = 0.0
+    samples = [(int(rng.integers(B)), int(rng.integers(W)), int(rng.integers(Hq))) for _ in range(n_attn)]
+    samples += [(0, 0, 0), (B - 1, W - 1, Hq - 1), (int(np.argmax(inp["prefix_len"])), W - 1, 0),
+                (int(np.argmin(inp["prefix_len"])), 0, Hq - 1)]
+    for (b, i, h) in samples:
+        want = orc.window_attention_row(inp["q"], inp["k"], inp["v"], inp["k_cache"], inp["v_cache"],
+                                        inp["block_table"], inp["prefix_len"], ref["pos_ids"], b, i, h,
+                                        theta=cfg.rope_theta)
+        err = float(np.abs(got[b, i, h] - want).max() / np.abs(want).max())
+        worst = max(worst, err)
+        assert err <= pu.ATTN_REL_TOL, (b, i, h, err)
+    print(cfg_name, impl, "worst sampled attention error", worst, "excluded sequences", excluded)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_cfg3_batched_serving_full_size_sampled(impl):
+    _sampled_full_size("cfg3_batched", impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_cfg4_long_context_full_size_sampled(impl):
+    _sampled_full_size("cfg4_long", impl)
