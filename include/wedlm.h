@@ -47,6 +47,7 @@ extern "C" {
 #define WEDLM_ERR_WORKSPACE_TOO_SMALL (-3)
 #define WEDLM_ERR_CUDA                (-4)
 #define WEDLM_ERR_TIMEOUT             (-5)
+#define WEDLM_ERR_STATIC_SCRATCH      (-6)  /* problem too large for the built-in scratch array */
 
 /* bits OR-ed into the device status word */
 #define WEDLM_STATUS_BAD_PAGE     1   /* block_table entry outside [0, num_pages)            */
@@ -197,6 +198,36 @@ int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const
                             int32_t* committed_tokens, int32_t* committed_count,
                             int32_t* filled_count, void* workspace, size_t workspace_bytes,
                             void* stream);
+
+/*
+ * wedlm_confidence_commit without a workspace argument, for hosts that must not allocate device
+ * memory while they run.  (The paper has no counterpart to this call; it exists for deployment.)
+ *
+ * Who needs it: a serving process that gave nearly all of HBM to its KV-cache pool when it started,
+ * so that a later cudaMalloc may fail and in any case stalls the device; or a decode loop that bans
+ * allocator calls after warm-up.  Such a caller passes inputs and outputs exactly as for
+ * wedlm_confidence_commit; the per-chunk partials go to an array of WEDLM_STATIC_SCRATCH_BYTES that
+ * is part of the library image.  Every GPU context that loads the library holds that array until the
+ * process exits.
+ *
+ *   - Limit: wedlm_confidence_workspace_bytes(cfg) must not exceed WEDLM_STATIC_SCRATCH_BYTES
+ *     (4 MiB = 262144 chunk partials; batch*window*ceil(vocab/8192) for bf16, /4096 for fp32).
+ *     Larger problems return WEDLM_ERR_STATIC_SCRATCH and launch nothing.
+ *   - The first call on each device looks up the array's device address (one runtime query, no
+ *     allocation) with that device current; make that first call before starting any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the previous call left there;
+ *     this routine needs none of it zeroed.  Two calls whose kernels can overlap on the GPU (different
+ *     streams, no ordering between them) race on the array: serialise them.
+ *   - The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ */
+#define WEDLM_STATIC_SCRATCH_BYTES (4u << 20)
+int wedlm_confidence_commit_static(const wedlm_config_t* cfg, const void* logits, const int32_t* perm,
+                                   const int32_t* n_filled, const int32_t* n_commit,
+                                   int32_t* window_tokens, uint8_t* filled, int32_t* prefix_len,
+                                   int32_t* window_len, int32_t* remaining_budget,
+                                   int32_t* argmax, float* maxprob, float* entropy, float* lse,
+                                   int32_t* committed_tokens, int32_t* committed_count,
+                                   int32_t* filled_count, void* stream);
 
 /*
  * Commit + shift + Refill of Algorithm 1 alone, for callers that did the selection themselves

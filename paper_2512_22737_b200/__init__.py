@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     load_library,
     make_config,
     wedlm_confidence_commit,
+    wedlm_confidence_commit_static,
     wedlm_confidence_workspace_bytes,
     wedlm_kv_append,
     wedlm_launch_count,

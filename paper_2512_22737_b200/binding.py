@@ -87,6 +87,9 @@ def load_library() -> ctypes.CDLL:
     lib.wedlm_confidence_commit.argtypes = [cfgp, vp, i32p, i32p, i32p, i32p, u8p, i32p, i32p, i32p,
                                             i32p, f32p, f32p, f32p, i32p, i32p, i32p, vp,
                                             ctypes.c_size_t, vp]
+    lib.wedlm_confidence_commit_static.restype = ctypes.c_int
+    lib.wedlm_confidence_commit_static.argtypes = [cfgp, vp, i32p, i32p, i32p, i32p, u8p, i32p, i32p, i32p,
+                                                   i32p, f32p, f32p, f32p, i32p, i32p, i32p, vp]
     lib.wedlm_window_refill.restype = ctypes.c_int
     lib.wedlm_window_refill.argtypes = [cfgp, i32p, i32p, u8p, i32p, i32p, i32p, i32p, i32p, vp]
     _lib = lib
@@ -213,6 +216,30 @@ def wedlm_confidence_commit(cfg, logits, perm, n_filled, n_commit, window_tokens
         _ptr(committed_count, i32, "committed_count"), _ptr(filled_count, i32, "filled_count"),
         _ptr(workspace, None, "workspace"), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
         _stream(stream)), "wedlm_confidence_commit")
+
+
+WEDLM_STATIC_SCRATCH_BYTES = 4 << 20
+WEDLM_ERR_STATIC_SCRATCH = -6
+
+
+def wedlm_confidence_commit_static(cfg, logits, perm, n_filled, n_commit, window_tokens, filled, prefix_len,
+                                   window_len, remaining_budget, argmax, maxprob, entropy, lse,
+                                   committed_tokens, committed_count, filled_count, stream=None) -> None:
+    """wedlm_confidence_commit for callers that may not allocate device memory (a process whose HBM is
+    already committed to a cache pool, a loop that bans allocator calls): same inputs and outputs, no
+    workspace; the scratch is a fixed 4 MiB array inside the library.  Raises WedlmError with code
+    WEDLM_ERR_STATIC_SCRATCH when batch*window*chunks does not fit.  Calls that may overlap on the GPU
+    must be serialised by the caller; the first call on a device should precede any stream capture."""
+    i32, u8, f32 = torch.int32, torch.uint8, torch.float32
+    _check(load_library().wedlm_confidence_commit_static(
+        ctypes.byref(cfg), _ptr(logits, cfg.torch_dtype, "logits"), _ptr(perm, i32, "perm"),
+        _ptr(n_filled, i32, "n_filled"), _ptr(n_commit, i32, "n_commit"),
+        _ptr(window_tokens, i32, "window_tokens"), _ptr(filled, u8, "filled"), _ptr(prefix_len, i32, "prefix_len"),
+        _ptr(window_len, i32, "window_len"), _ptr(remaining_budget, i32, "remaining_budget"),
+        _ptr(argmax, i32, "argmax"), _ptr(maxprob, f32, "maxprob"), _ptr(entropy, f32, "entropy"),
+        _ptr(lse, f32, "lse"), _ptr(committed_tokens, i32, "committed_tokens"),
+        _ptr(committed_count, i32, "committed_count"), _ptr(filled_count, i32, "filled_count"),
+        _stream(stream)), "wedlm_confidence_commit_static")
 
 
 def wedlm_window_refill(cfg, n_commit, window_tokens, filled, prefix_len, window_len, remaining_budget,

@@ -98,6 +98,7 @@ const char* wedlm_strerror(int code) {
     case WEDLM_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case WEDLM_ERR_CUDA: return "CUDA error";
     case WEDLM_ERR_TIMEOUT: return "device wait expired";
+    case WEDLM_ERR_STATIC_SCRATCH: return "problem too large for the built-in scratch array";
     default: return "unknown error code";
   }
 }

@@ -346,3 +346,60 @@ int launch_window_refill(const Shape& s, const wedlm_config_t* cfg, const int32_
 }
 
 }  // namespace wedlm
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant of wedlm_confidence_commit.
+//
+// Some hosts of this library may not allocate device memory once they are running: a serving
+// engine that has handed practically all of HBM to its KV-cache pool at start-up (a later cudaMalloc
+// can fail, and it synchronises the device), or a decode loop with a "no allocator calls after
+// warm-up" rule.  For them the chunk partials live in a fixed array inside the library image.
+// ------------------------------------------------------------------------------------------------
+#include <mutex>
+
+namespace {
+
+// Lives in every GPU context that loads the library, from load until process exit.
+static __device__ __align__(256) unsigned char g_conf_static_scratch[WEDLM_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+
+// In host code the array's name is only a handle; the address a kernel can use has to be asked for,
+// once per device, with that device current.
+int static_scratch_address(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return WEDLM_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (g_static_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_conf_static_scratch);
+    if (e != cudaSuccess || p == nullptr) return WEDLM_ERR_CUDA;
+    g_static_ptr[dev] = p;
+  }
+  *out = g_static_ptr[dev];
+  return WEDLM_OK;
+}
+
+}  // namespace
+
+extern "C" int wedlm_confidence_commit_static(const wedlm_config_t* cfg, const void* logits, const int32_t* perm,
+                                              const int32_t* n_filled, const int32_t* n_commit,
+                                              int32_t* window_tokens, uint8_t* filled, int32_t* prefix_len,
+                                              int32_t* window_len, int32_t* remaining_budget, int32_t* argmax,
+                                              float* maxprob, float* entropy, float* lse,
+                                              int32_t* committed_tokens, int32_t* committed_count,
+                                              int32_t* filled_count, void* stream) {
+  const size_t need = wedlm_confidence_workspace_bytes(cfg);     // 0 for a NULL / invalid config
+  if (need == 0) return WEDLM_ERR_INVALID_ARG;
+  if (need > (size_t)WEDLM_STATIC_SCRATCH_BYTES) return WEDLM_ERR_STATIC_SCRATCH;
+  void* scratch = nullptr;
+  int rc = static_scratch_address(&scratch);
+  if (rc != WEDLM_OK) return rc;
+  // Every partial that pass 2 reads is written by pass 1 of the same call, so nothing in the array
+  // has to start at zero and the previous call's contents are harmless.
+  return wedlm_confidence_commit(cfg, logits, perm, n_filled, n_commit, window_tokens, filled, prefix_len, window_len,
+                                 remaining_budget, argmax, maxprob, entropy, lse, committed_tokens, committed_count,
+                                 filled_count, scratch, (size_t)WEDLM_STATIC_SCRATCH_BYTES, stream);
+}
