@@ -1,5 +1,6 @@
 // C ABI of the WeDLM step library: argument validation, workspace planning, kernel dispatch.
 #include <atomic>
+#include <cstdlib>
 
 #include "common.cuh"
 
@@ -64,15 +65,31 @@ namespace wedlm {
 AttnPlan plan_attention(const wedlm_config_t* c) {
   AttnPlan p{};
   const int elem = c->dtype == WEDLM_DTYPE_BF16 ? 2 : 4;
-  p.impl = WEDLM_ATTN_GENERIC;
   const long long total = (long long)c->max_prefix_len + c->window;
-  const long long n_rb = (c->window + 15) / 16;
-  const long long units = (long long)c->batch * c->n_q_heads * n_rb;
-  long long want = units > 0 ? (148LL * 4 + units - 1) / units : 1;      // a few blocks per SM
-  long long cap = total / 256 > 1 ? total / 256 : 1;                      // keep chunks >= 256 keys
-  long long S = want < 1 ? 1 : (want > cap ? cap : want);
-  long long chunk = (total + S - 1) / S;
-  chunk = (chunk + c->page_size - 1) / c->page_size * c->page_size;
+  const bool tensor_ok = attn_tensor_supported(c);
+  p.impl = (c->attn_impl == WEDLM_ATTN_GENERIC || !tensor_ok) ? WEDLM_ATTN_GENERIC : WEDLM_ATTN_TENSOR;
+  long long S, chunk;
+  if (p.impl == WEDLM_ATTN_TENSOR) {
+    // one CTA per (sequence, kv head, 128-row tile, key chunk); two CTAs per SM.  Split the keys
+    // only as far as needed to give every CTA slot a few work items; chunks are whole 64-key tiles.
+    const int G = c->n_q_heads / c->n_kv_heads;
+    const long long w_t = 128 / G;
+    const long long units = (long long)c->batch * c->n_kv_heads * ((c->window + w_t - 1) / w_t);
+    long long want = units > 0 ? (3LL * 296 + units - 1) / units : 1;
+    if (const char* e = getenv("WEDLM_ATTN_SPLITS")) { long long v = atoll(e); if (v > 0) want = v; }
+    long long cap = total / 1024 > 1 ? total / 1024 : 1;                    // keep chunks >= 1024 keys
+    S = want < 1 ? 1 : (want > cap ? cap : want);
+    chunk = (total + S - 1) / S;
+    chunk = (chunk + 63) / 64 * 64;
+  } else {
+    const long long n_rb = (c->window + 15) / 16;
+    const long long units = (long long)c->batch * c->n_q_heads * n_rb;
+    long long want = units > 0 ? (148LL * 4 + units - 1) / units : 1;      // a few blocks per SM
+    long long cap = total / 256 > 1 ? total / 256 : 1;                      // keep chunks >= 256 keys
+    S = want < 1 ? 1 : (want > cap ? cap : want);
+    chunk = (total + S - 1) / S;
+    chunk = (chunk + c->page_size - 1) / c->page_size * c->page_size;
+  }
   S = (total + chunk - 1) / chunk;
   p.n_splits = (int)S;
   p.chunk = (int)chunk;
@@ -143,6 +160,7 @@ int wedlm_window_attn(const wedlm_config_t* cfg, const void* q, const void* k, c
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(k_cache) || !aligned16(v_cache) ||
       !aligned16(out) || !aligned16(workspace))
     return WEDLM_ERR_INVALID_ARG;
+  if (cfg->attn_impl == WEDLM_ATTN_TENSOR && !attn_tensor_supported(cfg)) return WEDLM_ERR_UNSUPPORTED;
   AttnPlan plan = plan_attention(cfg);
   if (workspace_bytes < plan.total_bytes) return WEDLM_ERR_WORKSPACE_TOO_SMALL;
   Shape s = make_shape(cfg);
@@ -157,7 +175,10 @@ int wedlm_window_attn(const wedlm_config_t* cfg, const void* q, const void* k, c
   cudaEvent_t ev0 = t_ev_before, ev1 = t_ev_after;
   t_ev_before = t_ev_after = nullptr;
   if (ev0 && cudaEventRecord(ev0, st) != cudaSuccess) return WEDLM_ERR_CUDA;
-  rc = launch_attn_generic(s, plan, q_rot, k_cache, v_cache, block_table, prefix_len, out, part_o, part_ml, status, st);
+  if (plan.impl == WEDLM_ATTN_TENSOR)
+    rc = launch_attn_tensor(s, plan, q_rot, k_cache, v_cache, block_table, prefix_len, out, part_o, part_ml, status, st);
+  else
+    rc = launch_attn_generic(s, plan, q_rot, k_cache, v_cache, block_table, prefix_len, out, part_o, part_ml, status, st);
   if (ev1 && cudaEventRecord(ev1, st) != cudaSuccess) return WEDLM_ERR_CUDA;
   if (rc != WEDLM_OK) return rc;
   if (plan.n_splits > 1) rc = launch_attn_merge(s, plan, prefix_len, part_o, part_ml, out, st);

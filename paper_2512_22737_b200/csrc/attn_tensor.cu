@@ -1,0 +1,546 @@
+// Window attention on the 5th-generation tensor cores (sm_100a): TMA-staged K/V pages, tcgen05.mma
+// with accumulators in tensor memory, online softmax in registers.
+//
+// What it computes (Section 5.2, "a causal forward over the current window conditioned on the cached
+// prefix"): for one (sequence b, KV head g) the M = W_t*G query rows (W_t window slots x G grouped
+// query heads, G*W_t = 128) attend to cache positions 0..P-1 and to the staged window rows P..P+i
+// (physical row i sees window rows j <= i).  All keys are read from the paged cache: the window's
+// rotated K and V were staged there by the RoPE/stage kernel before this kernel starts.
+//
+// One CTA = one (b, g, 128-row tile, key chunk).  Warps 0-3 (128 threads, one query row each) run the
+// online softmax; warp 4 lane 0 issues every TMA copy and every MMA.  Per 64-key tile:
+//     S[t&1] = Q K_t^T   (tcgen05.mma, 8 k-steps, fp32 in TMEM columns 0..127, double buffered)
+//     softmax threads: tcgen05.ld S row -> mask -> running max (lazy rescale) -> p = 2^(s*c - m*c)
+//                      -> bf16 P tile into shared memory (128-byte swizzle)
+//     O += P V_t         (tcgen05.mma, 4 k-steps, V consumed MN-major straight from its page layout)
+// Two CTAs fit on an SM (112 KB shared memory, 256 TMEM columns each), so one CTA's softmax overlaps
+// the other's MMAs and loads.  Every wait on an mbarrier is bounded; on expiry the CTA records
+// WEDLM_STATUS_WAIT_EXPIRED, drains its copies, frees its tensor memory and returns.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <math_constants.h>
+
+#include "common.cuh"
+
+namespace wedlm {
+namespace {
+
+constexpr int kTileN = 64;            // keys per tile (4 pages)
+constexpr int kD = 128;               // head size
+constexpr int kPage = 16;
+constexpr int kPagesPerTile = kTileN / kPage;
+constexpr int kThreadsT = 160;        // 4 softmax warps + 1 issue warp
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr float kLazyRescaleLog2 = 8.0f;   // keep the old reference while the max grew by < 2^8
+
+// shared memory map (bytes, base 1024-aligned)
+constexpr uint32_t kOffQ = 0;                       // 2 halves x [128 rows x 128 B]
+constexpr uint32_t kOffK = 32768;                   // 2 stages x 2 halves x [64 rows x 128 B]
+constexpr uint32_t kOffV = 65536;                   // 2 stages x 2 halves x [64 rows x 128 B]
+constexpr uint32_t kOffP = 98304;                   // [128 rows x 128 B] bf16 probabilities
+constexpr uint32_t kOffBar = 114688;
+constexpr uint32_t kSmemBytes = kOffBar + 256;
+constexpr uint32_t kStageBytes = 16384;
+constexpr uint32_t kHalfKV = 8192;
+constexpr uint32_t kHalfQ = 16384;
+
+enum Bar { Q_FULL = 0, K_FULL0, K_FULL1, V_FULL0, V_FULL1, S_FULL0, S_FULL1, O_DONE, P_READY, N_BARS };
+
+struct TensorAttnParams {
+  int B, W, Hq, Hkv, G, W_t, n_mtiles, n_splits, chunk, max_pages, num_pages;
+  float scale_log2;          // softmax scale * log2(e)
+  const int32_t* block_table;
+  const int32_t* prefix_len;
+  __nv_bfloat16* out;
+  float* part_o;
+  float* part_ml;
+  int32_t* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within the spin limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
+// K-major operand: rows of 128 B, 8-row groups 1024 B apart (SBO); LBO unused.
+// MN-major operand (V as B of P*V): 64-element blocks along N are `lbo` bytes apart, 8-key groups 1024 B.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(lbo_bytes >> 4) << 16;
+  d |= (uint64_t)(sbo_bytes >> 4) << 32;
+  d |= 1ull << 46;
+  d |= 2ull << 61;
+  return d;
+}
+
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(128 >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// grid: x = split * n_mtiles + mtile, y = kv head, z = sequence
+__global__ void __launch_bounds__(kThreadsT, 2)
+attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                   const __grid_constant__ CUtensorMap tm_v, const TensorAttnParams p) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int split = blockIdx.x / p.n_mtiles, mtile = blockIdx.x - split * p.n_mtiles;
+  const int g = blockIdx.y, b = blockIdx.z;
+
+  int P = p.prefix_len[b];
+  if (P < 0) { if (p.status && tid == 0) atomicOr(p.status, WEDLM_STATUS_BAD_LENGTH); P = 0; }
+  const int total = P + p.W;
+  const int n_valid = (total + p.chunk - 1) / p.chunk;
+  if (split >= n_valid) return;
+  const int slot0 = mtile * p.W_t;                          // first window slot of this row tile
+  const int slot_end = min(p.W, slot0 + p.W_t);
+  const int kv_begin = split * p.chunk;
+  const int kv_end = min(min(kv_begin + p.chunk, total), P + slot_end);   // horizon of the last row
+  const int T = kv_begin < kv_end ? (kv_end - kv_begin + kTileN - 1) / kTileN : 0;
+
+  // this thread's query row (softmax warps only)
+  const int r = tid;                                         // row of the 128-row tile
+  const int i_row = slot0 + r / p.G;                         // physical window slot
+  const int h = g * p.G + r % p.G;                           // query head
+  const bool row_valid = (tid < 128) && (i_row < p.W);
+  const float c = p.scale_log2;
+
+  if (T == 0) {
+    // nothing visible in this chunk for these rows: an empty partial (only possible when n_splits > 1)
+    if (row_valid && p.n_splits > 1) {
+      const size_t prow = (((size_t)b * p.Hq + h) * p.W + i_row) * p.n_splits + split;
+      float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+      float4* dst = reinterpret_cast<float4*>(p.part_o + prow * kD);
+      for (int d4 = 0; d4 < kD / 4; ++d4) dst[d4] = z;
+      p.part_ml[prow * 2] = -CUDART_INF_F;
+      p.part_ml[prow * 2 + 1] = 0.f;
+    }
+    return;
+  }
+
+  const uint32_t sbase = smem_u32(smem);
+  if ((sbase & 1023u) != 0u) {     // the swizzled layouts need a 1024-byte aligned base
+    if (p.status && tid == 0) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
+    return;
+  }
+  const uint32_t bars = sbase + kOffBar;
+  auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kOffBar + 8 * N_BARS);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  if (tid == 0) {
+    for (int i = 0; i < N_BARS; ++i) mbar_init(bar(i), i == P_READY ? 128u : 1u);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32((const void*)tmem_slot)), "r"(256u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_S = tmem_base;            // columns [0,64) and [64,128)
+  const uint32_t tmem_O = tmem_base + 128u;     // columns [128,256)
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ issue warp (one lane)
+    if (lane == 0) {
+      bool ok = true;
+      const uint32_t idesc_qk = make_idesc(kTileN, false);
+      const uint32_t idesc_pv = make_idesc(kD, true);
+      const int oob_row = p.num_pages * p.Hkv * kPage;      // a row coordinate past the end: zero fill
+
+      auto page_row = [&](int key0) -> int {
+        const int lp = key0 / kPage;
+        int pp = -1;
+        if (lp < p.max_pages) pp = p.block_table[(size_t)b * p.max_pages + lp];
+        if (pp < 0 || pp >= p.num_pages) {
+          if (key0 < kv_end && p.status) atomicOr(p.status, lp < p.max_pages ? WEDLM_STATUS_BAD_PAGE : WEDLM_STATUS_BAD_LENGTH);
+          return oob_row;
+        }
+        return (pp * p.Hkv + g) * kPage;
+      };
+      auto load_tile = [&](const CUtensorMap* map, uint32_t dst_stage, uint32_t full_bar, int t) {
+        mbar_expect_tx(full_bar, kStageBytes);
+#pragma unroll
+        for (int pg = 0; pg < kPagesPerTile; ++pg) {
+          const int y = page_row(kv_begin + t * kTileN + pg * kPage);
+          tma_load_2d(dst_stage + pg * 2048u, map, 0, y, full_bar);
+          tma_load_2d(dst_stage + kHalfKV + pg * 2048u, map, 64, y, full_bar);
+        }
+      };
+
+      // Q tile: two 64-element halves of [W_t slots x G heads] rows
+      const int q_slots = min(p.W_t, p.W);        // box height along the window dimension
+      mbar_expect_tx(bar(Q_FULL), (uint32_t)(2 * 64 * p.G * q_slots * 2));
+      tma_load_4d(sbase + kOffQ, &tm_q, 0, g * p.G, slot0, b, bar(Q_FULL));
+      tma_load_4d(sbase + kOffQ + kHalfQ, &tm_q, 64, g * p.G, slot0, b, bar(Q_FULL));
+      for (int t = 0; t < 2 && t < T; ++t) {
+        load_tile(&tm_k, sbase + kOffK + t * kStageBytes, bar(K_FULL0 + t), t);
+        load_tile(&tm_v, sbase + kOffV + t * kStageBytes, bar(V_FULL0 + t), t);
+      }
+      auto issue_qk = [&](int t) {
+        const uint32_t st = (uint32_t)t & 1u;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint64_t ad = make_desc(sbase + kOffQ + (kk >> 2) * kHalfQ + (kk & 3) * 32u, 16u, 1024u);
+          const uint64_t bd = make_desc(sbase + kOffK + st * kStageBytes + (kk >> 2) * kHalfKV + (kk & 3) * 32u, 16u, 1024u);
+          umma(tmem_S + st * 64u, ad, bd, idesc_qk, kk > 0);
+        }
+        umma_commit(bar(S_FULL0 + st));
+      };
+
+      ok = mbar_wait(bar(Q_FULL), 0);
+      if (ok) ok = mbar_wait(bar(K_FULL0), 0);
+      if (ok) issue_qk(0);
+      for (int t = 0; ok && t < T; ++t) {
+        const uint32_t st = (uint32_t)t & 1u, ph = ((uint32_t)t >> 1) & 1u;
+        if (t + 1 < T) {
+          // S[(t+1)&1] was last read by the softmax of tile t-1, whose P_READY we saw one iteration ago
+          const uint32_t st1 = st ^ 1u, ph1 = ((uint32_t)(t + 1) >> 1) & 1u;
+          ok = mbar_wait(bar(K_FULL0 + st1), ph1);
+          if (!ok) break;
+          issue_qk(t + 1);
+        }
+        if (t + 2 < T) {
+          // K stage st is free once Q K_t^T has completed
+          ok = mbar_wait(bar(S_FULL0 + st), ph);
+          if (!ok) break;
+          load_tile(&tm_k, sbase + kOffK + st * kStageBytes, bar(K_FULL0 + st), t + 2);
+        }
+        ok = mbar_wait(bar(P_READY), (uint32_t)t & 1u);
+        if (!ok) break;
+        ok = mbar_wait(bar(V_FULL0 + st), ph);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint64_t ad = make_desc(sbase + kOffP + j * 32u, 16u, 1024u);
+          const uint64_t bd = make_desc(sbase + kOffV + st * kStageBytes + j * 2048u, kHalfKV, 1024u);
+          umma(tmem_O, ad, bd, idesc_pv, (t > 0) || (j > 0));
+        }
+        umma_commit(bar(O_DONE));
+        if (t + 2 < T) {
+          // V stage st is free once P V_t has completed
+          ok = mbar_wait(bar(O_DONE), (uint32_t)t & 1u);
+          if (!ok) break;
+          load_tile(&tm_v, sbase + kOffV + st * kStageBytes, bar(V_FULL0 + st), t + 2);
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        if (p.status) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax warps: one row per thread
+    const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+    const int limit = row_valid ? P + i_row : -1;           // last visible key index (inclusive)
+    float m_ref = -CUDART_INF_F;                            // reference maximum (raw score units)
+    float l = 0.f;
+    bool ok = true;
+    for (int t = 0; t < T; ++t) {
+      const uint32_t st = (uint32_t)t & 1u, ph = ((uint32_t)t >> 1) & 1u;
+      ok = mbar_wait(bar(S_FULL0 + st), ph);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t raw[64];
+      {
+        uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&raw[0]);
+        uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&raw[32]);
+        tmem_ld32(tmem_S + lane_sel + st * 64u, lo);
+        tmem_ld32(tmem_S + lane_sel + st * 64u + 32u, hi);
+        tmem_wait_ld();
+      }
+      float s[64];
+      const int tile0 = kv_begin + t * kTileN;
+      const bool need_mask = tile0 + kTileN > min(P + slot0 + 1, kv_end);   // block-uniform
+      float m_tile = -CUDART_INF_F;
+      if (need_mask) {
+#pragma unroll
+        for (int cc = 0; cc < 64; ++cc) {
+          const int key = tile0 + cc;
+          float x = __uint_as_float(raw[cc]);
+          x = (key <= limit && key < kv_end) ? x : -CUDART_INF_F;
+          s[cc] = x;
+          m_tile = fmaxf(m_tile, x);
+        }
+      } else {
+#pragma unroll
+        for (int cc = 0; cc < 64; ++cc) {
+          s[cc] = __uint_as_float(raw[cc]);
+          m_tile = fmaxf(m_tile, s[cc]);
+        }
+      }
+      // lazy reference: only move it when the maximum grew by more than 2^kLazyRescaleLog2
+      float alpha = 1.f;
+      bool moved = false;
+      if (m_tile > -CUDART_INF_F && (m_ref == -CUDART_INF_F || (m_tile - m_ref) * c > kLazyRescaleLog2)) {
+        alpha = (m_ref == -CUDART_INF_F) ? 0.f : exp2f((m_ref - m_tile) * c);
+        m_ref = m_tile;
+        moved = true;
+      }
+      const float neg_mc = (m_ref == -CUDART_INF_F) ? 0.f : -m_ref * c;
+      float sum = 0.f;
+      uint32_t pk[32];
+#pragma unroll
+      for (int cc = 0; cc < 64; cc += 2) {
+        const float p0 = exp2f(fmaf(s[cc], c, neg_mc));
+        const float p1 = exp2f(fmaf(s[cc + 1], c, neg_mc));
+        sum += p0 + p1;
+        pk[cc >> 1] = pack_bf16(p0, p1);
+      }
+      l = l * alpha + sum;
+      // P buffer and O are free / stable once P V_{t-1} has completed
+      if (t > 0) {
+        ok = mbar_wait(bar(O_DONE), (uint32_t)(t - 1) & 1u);
+        if (!ok) break;
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, moved)) {
+#pragma unroll 1
+          for (int ch = 0; ch < 4; ++ch) {
+            uint32_t o[32];
+            tmem_ld32(tmem_O + lane_sel + ch * 32u, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(tmem_O + lane_sel + ch * 32u, o);
+          }
+          tmem_wait_st();
+        }
+      }
+      // bf16 P row into the 128-byte-swizzled K-major tile: 16-byte chunk j of row r sits at j ^ (r & 7)
+      {
+        uint8_t* prow = smem + kOffP + r * 128;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          uint4 v = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+          *reinterpret_cast<uint4*>(prow + ((j ^ (r & 7)) << 4)) = v;
+        }
+      }
+      // last tile: V rows of keys beyond the horizon may hold anything (0 * NaN = NaN): zero them
+      if (t == T - 1 && kv_end - tile0 < kTileN) {
+        ok = mbar_wait(bar(V_FULL0 + st), ph);
+        if (!ok) break;
+        const int first_bad = kv_end - tile0;
+        uint8_t* vst = smem + kOffV + st * kStageBytes;
+        for (int idx = tid; idx < (kTileN - first_bad) * 16; idx += 128) {      // 16 x 16-byte chunks per key row
+          const int row = first_bad + idx / 16, ch = idx % 16;
+          *reinterpret_cast<uint4*>(vst + (ch >> 3) * kHalfKV + row * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      fence_async_smem();
+      tc_fence_before();
+      mbar_arrive(bar(P_READY));
+    }
+    if (ok) ok = mbar_wait(bar(O_DONE), (uint32_t)(T - 1) & 1u);
+    if (!ok) {
+      *abort_flag = 1;
+      if (p.status) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
+    } else {
+      tc_fence_after();
+      const bool final_out = p.n_splits == 1;
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      const size_t orow = (((size_t)b * p.W + i_row) * p.Hq + h) * kD;
+      const size_t prow = (((size_t)b * p.Hq + h) * p.W + i_row) * p.n_splits + split;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t o[32];
+        tmem_ld32(tmem_O + lane_sel + ch * 32u, o);
+        tmem_wait_ld();
+        if (!row_valid) continue;
+        if (final_out) {
+          uint4* dst = reinterpret_cast<uint4*>(p.out + orow + ch * 32);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(o[8 * q4 + 0]) * inv, __uint_as_float(o[8 * q4 + 1]) * inv);
+            v.y = pack_bf16(__uint_as_float(o[8 * q4 + 2]) * inv, __uint_as_float(o[8 * q4 + 3]) * inv);
+            v.z = pack_bf16(__uint_as_float(o[8 * q4 + 4]) * inv, __uint_as_float(o[8 * q4 + 5]) * inv);
+            v.w = pack_bf16(__uint_as_float(o[8 * q4 + 6]) * inv, __uint_as_float(o[8 * q4 + 7]) * inv);
+            dst[q4] = v;
+          }
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(p.part_o + prow * kD + ch * 32);
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4) dst[q4] = make_uint4(o[4 * q4], o[4 * q4 + 1], o[4 * q4 + 2], o[4 * q4 + 3]);
+        }
+      }
+      if (row_valid && !final_out) {
+        p.part_ml[prow * 2] = (m_ref == -CUDART_INF_F) ? -CUDART_INF_F : m_ref * c;     // log2 domain
+        p.part_ml[prow * 2 + 1] = l;
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag != 0) {
+    // a wait expired: give copies that may still be in flight a bounded time (about 0.2 ms) to land
+    // before this CTA's shared memory is handed to another CTA
+    for (int it = 0; it < 200; ++it) __nanosleep(1000);
+  }
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- host
+PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  if (fn) return fn;
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
+  return fn;
+}
+
+}  // namespace
+
+bool attn_tensor_supported(const wedlm_config_t* c) {
+  if (c->dtype != WEDLM_DTYPE_BF16 || c->head_dim != kD || c->page_size != kPage) return false;
+  const int G = c->n_q_heads / c->n_kv_heads;
+  if (G < 1 || G > 128 || (128 % G) != 0) return false;
+  if ((long long)c->num_pages * c->n_kv_heads * kPage >= (1ll << 31)) return false;
+  return true;
+}
+
+int launch_attn_tensor(const Shape& s, const AttnPlan& plan, const void* q_rot, const void* k_cache,
+                       const void* v_cache, const int32_t* block_table, const int32_t* prefix_len, void* out,
+                       float* part_o, float* part_ml, int32_t* status, cudaStream_t st) {
+  auto encode = get_encode();
+  if (!encode) return WEDLM_ERR_CUDA;
+  const int W_t = 128 / s.G;
+  const int n_mtiles = (s.W + W_t - 1) / W_t;
+
+  CUtensorMap tm_q, tm_k, tm_v;
+  {
+    // q_rot [B][W][Hq][D] as a 4-D tensor (D, Hq, W, B); box = (64, G, min(W_t, W), 1)
+    cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)s.Hq, (cuuint64_t)s.W, (cuuint64_t)s.B};
+    cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)s.Hq * kD * 2, (cuuint64_t)s.W * s.Hq * kD * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)s.G, (cuuint32_t)(W_t < s.W ? W_t : s.W), 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (encode(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q_rot), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return WEDLM_ERR_CUDA;
+  }
+  for (int which = 0; which < 2; ++which) {
+    // cache [num_pages][Hkv][16][D] as a 2-D tensor (D, rows); box = one page of one head, 64 elements wide
+    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)s.num_pages * s.Hkv * kPage};
+    cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kPage};
+    cuuint32_t estr[2] = {1, 1};
+    if (encode(which ? &tm_v : &tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(which ? v_cache : k_cache),
+               dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return WEDLM_ERR_CUDA;
+  }
+  TensorAttnParams p;
+  p.B = s.B; p.W = s.W; p.Hq = s.Hq; p.Hkv = s.Hkv; p.G = s.G; p.W_t = W_t; p.n_mtiles = n_mtiles;
+  p.n_splits = plan.n_splits; p.chunk = plan.chunk; p.max_pages = s.max_pages; p.num_pages = s.num_pages;
+  p.scale_log2 = s.scale * 1.4426950408889634f;
+  p.block_table = block_table; p.prefix_len = prefix_len;
+  p.out = (__nv_bfloat16*)out; p.part_o = part_o; p.part_ml = part_ml; p.status = status;
+
+  // per device; cheap enough to repeat on every launch
+  if (cudaFuncSetAttribute(attn_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
+    return WEDLM_ERR_CUDA;
+  dim3 grid(plan.n_splits * n_mtiles, s.Hkv, s.B);
+  attn_tensor_kernel<<<grid, kThreadsT, kSmemBytes, st>>>(tm_q, tm_k, tm_v, p);
+  count_launch();
+  return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace wedlm

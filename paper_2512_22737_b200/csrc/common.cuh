@@ -66,6 +66,11 @@ int launch_attn_generic(const Shape& s, const AttnPlan& plan, const void* q_rot,
                         const void* v_cache, const int32_t* block_table, const int32_t* prefix_len, void* out,
                         float* part_o, float* part_ml, int32_t* status, cudaStream_t st);
 
+bool attn_tensor_supported(const wedlm_config_t* cfg);
+int launch_attn_tensor(const Shape& s, const AttnPlan& plan, const void* q_rot, const void* k_cache,
+                       const void* v_cache, const int32_t* block_table, const int32_t* prefix_len, void* out,
+                       float* part_o, float* part_ml, int32_t* status, cudaStream_t st);
+
 int launch_attn_merge(const Shape& s, const AttnPlan& plan, const int32_t* prefix_len, const float* part_o,
                       const float* part_ml, void* out, cudaStream_t st);
 

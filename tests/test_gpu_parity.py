@@ -12,7 +12,7 @@ from oracle import wedlm_oracle as orc
 
 pytestmark = pytest.mark.gpu
 
-IMPLS = ["generic"]
+IMPLS = ["generic", "tensor"]
 
 
 def _small_qwen(**kw):
@@ -113,6 +113,54 @@ def test_unaligned_vocab_takes_the_scalar_path():
     import parity_util as pu
     cfg = _small_qwen(batch=2, window=8, prefix_lo=20, prefix_hi=20, vocab=10007, boost=11.0, name="oddvocab")
     pu.full_parity(cfg, make_step(cfg, seed=41))
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("W,P", [(16, 100), (40, 333), (64, 64), (5, 1000), (1, 31), (32, 0), (33, 4097)])
+def test_window_sizes_and_row_tiles(impl, W, P):
+    """W*G below, equal to and above one 128-row tile, partial second tile, chunk boundaries."""
+    import parity_util as pu
+    cfg = _small_qwen(batch=2, window=W, prefix_lo=P, prefix_hi=P + 70, vocab=2048, name="rowtiles")
+    pu.full_parity(cfg, make_step(cfg, seed=W * 1000 + P), attn_impl=impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_stale_cache_rows_beyond_the_window_cannot_leak(impl):
+    """Rows of the last page past P + W may hold anything (here NaN and Inf bit patterns); they are
+    masked by index, so the outputs must not change."""
+    import parity_util as pu
+    cfg = _small_qwen(batch=2, window=8, prefix_lo=70, prefix_hi=70, vocab=2048, name="stale")
+    inp = make_step(cfg, seed=77)
+    ref = pu.oracle_step(cfg, inp)
+    B, W = inp["filled"].shape
+    for b in range(B):
+        P = int(inp["prefix_len"][b])
+        for t in range(P + W, ((P + W + 15) // 16) * 16):
+            pg = inp["block_table"][b, t // 16]
+            inp["k_cache"][pg, :, t % 16, :] = 0x7FC0       # NaN
+            inp["v_cache"][pg, :, t % 16, :] = 0x7F80       # +Inf
+    # every spare / unowned page too
+    owned = set(inp["block_table"][inp["block_table"] >= 0].tolist())
+    for pg in range(inp["k_cache"].shape[0]):
+        if pg not in owned:
+            inp["k_cache"][pg] = 0x7FC0
+            inp["v_cache"][pg] = 0x7FC0
+    step, d = pu.run_gpu_step(cfg, inp, attn_impl=impl)
+    got = pu.bf16_from_device(step.out)
+    assert np.isfinite(got).all()
+    assert pu.attn_vector_error(got, ref["out"]).max() <= pu.ATTN_REL_TOL
+
+
+def test_tensor_path_refuses_shapes_it_does_not_cover():
+    import paper_2512_22737_b200 as w
+    cfg = w.make_config(batch=1, window=8, n_q_heads=4, n_kv_heads=2, head_dim=64, max_pages_per_seq=8,
+                        num_pages=8, max_prefix_len=64, attn_impl="tensor")
+    t = torch.zeros(4096, dtype=torch.bfloat16, device="cuda")
+    i = torch.zeros(64, dtype=torch.int32, device="cuda")
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    with pytest.raises(w.WedlmError) as e:
+        w.wedlm_window_attn(cfg, t, t, t, t, t, i, i, i, t, None, ws)
+    assert e.value.code == -2
 
 
 def test_empty_batch_is_a_noop():
