@@ -196,11 +196,13 @@ class Workload:
     streams (cache, logits) when one copy would fit in L2, and one fresh copy of the small window
     state per iteration."""
 
-    def __init__(self, name, seed, attn_impl, n_state):
+    def __init__(self, name, seed, attn_impl, n_state, batch=None):
         import torch
         import paper_2512_22737_b200 as w
         from workloads import get_config, make_step
         self.cfg = get_config(name)
+        if batch:
+            self.cfg = self.cfg.replace(batch=batch)
         t0 = time.time()
         self.inp = make_step(self.cfg, seed=seed)
         log(f"[{name}] inputs drawn in {time.time() - t0:.1f}s")
@@ -348,7 +350,7 @@ def run_product(args):
 
     sampler = ClockSampler(local) if rank == 0 else None
     n_state = args.steps + args.warmup
-    wl = Workload(args.workload, BASE_SEED + rank, args.attn, n_state)
+    wl = Workload(args.workload, BASE_SEED + rank, args.attn, n_state, args.batch)
     if sampler:
         sampler.start()
 
@@ -371,7 +373,10 @@ def run_product(args):
         committed_total = float(committed)
     assert int(wl.step.status.item()) == 0, "device status word set during the benchmark"
 
-    e2e_ms, e2e_committed, h2d, d2h = time_e2e(wl, max(3, min(args.steps, 10)), 3, sampler)
+    if args.no_e2e:
+        e2e_ms, e2e_committed, h2d, d2h = float("nan"), 0, 0, 0
+    else:
+        e2e_ms, e2e_committed, h2d, d2h = time_e2e(wl, max(3, min(args.steps, 10)), 3, sampler)
     te = torch.tensor([e2e_ms, float(e2e_committed)], dtype=torch.float64, device="cuda")
     if world > 1:
         tm = te.clone()
@@ -401,7 +406,7 @@ def run_product(args):
                 others[name] = {"error": repr(e)}
     if sampler:
         sampler.stop()
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.no_cpu:
         cores = len(os.sched_getaffinity(0))
         n_s = min(wl.cfg.batch, 8 if wl.cfg.batch >= 8 else wl.cfg.batch)
         log(f"timing the oracle on {n_s} sequences ...")
@@ -420,7 +425,7 @@ def run_product(args):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.cfg.dtype == "bf16" else "f32",
             "data": "synthetic",
-            "config": {"workload": wl.cfg.name, "batch_per_gpu": wl.cfg.batch, "window": wl.cfg.window,
+            "config": {"workload": wl.cfg.name if not args.batch else f"{wl.cfg.name}@batch{args.batch}", "batch_per_gpu": wl.cfg.batch, "window": wl.cfg.window,
                        "prefix_tokens_per_gpu": int(wl.inp["prefix_len"].sum()), "attn_impl": args.attn,
                        "l2": "inputs_exceed_l2" if wl.n_copies == 1 else f"rotating_{wl.n_copies}_copies",
                        "committed_tokens_per_step": committed_total,
@@ -453,6 +458,9 @@ def main():
     ap.add_argument("--workload", default="cfg3_batched")
     ap.add_argument("--attn", default="auto", choices=["auto", "generic", "tensor"])
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary workloads")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing (profiling runs)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "product" else args.warmup
     if args.impl == "reference":

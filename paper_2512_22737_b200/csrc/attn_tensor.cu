@@ -8,7 +8,7 @@
 // rotated K and V were staged there by the RoPE/stage kernel before this kernel starts.
 //
 // One CTA = one (b, g, 128-row tile, key chunk).  Warps 0-3 (128 threads, one query row each) run the
-// online softmax; warp 4 lane 0 issues every TMA copy and every MMA.  Per 64-key tile:
+// online softmax; warp 4 lane 0 issues every MMA; warp 5 lane 0 issues every TMA copy.  Per 64-key tile:
 //     S[t&1] = Q K_t^T   (tcgen05.mma, 8 k-steps, fp32 in TMEM columns 0..127, double buffered)
 //     softmax threads: tcgen05.ld S row -> mask -> running max (lazy rescale) -> p = 2^(s*c - m*c)
 //                      -> bf16 P tile into shared memory (128-byte swizzle)
@@ -29,7 +29,7 @@ constexpr int kTileN = 64;            // keys per tile (4 pages)
 constexpr int kD = 128;               // head size
 constexpr int kPage = 16;
 constexpr int kPagesPerTile = kTileN / kPage;
-constexpr int kThreadsT = 160;        // 4 softmax warps + 1 issue warp
+constexpr int kThreadsT = 192;        // 4 softmax warps + MMA issue warp + TMA producer warp
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kLazyRescaleLog2 = 8.0f;   // keep the old reference while the max grew by < 2^8
 
@@ -44,7 +44,8 @@ constexpr uint32_t kStageBytes = 16384;
 constexpr uint32_t kHalfKV = 8192;
 constexpr uint32_t kHalfQ = 16384;
 
-enum Bar { Q_FULL = 0, K_FULL0, K_FULL1, V_FULL0, V_FULL1, S_FULL0, S_FULL1, O_DONE, P_READY, N_BARS };
+enum Bar { Q_FULL = 0, K_FULL0, K_FULL1, V_FULL0, V_FULL1, S_FULL0, S_FULL1, O_DONE, P_READY, K_FREE0, K_FREE1,
+           V_FREE0, V_FREE1, N_BARS };
 
 struct TensorAttnParams {
   int B, W, Hq, Hkv, G, W_t, n_mtiles, n_splits, chunk, max_pages, num_pages;
@@ -206,7 +207,7 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   }
   const uint32_t bars = sbase + kOffBar;
   auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kOffBar + 8 * N_BARS);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kOffBar + 112);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   if (tid == 0) {
@@ -227,42 +228,13 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const uint32_t tmem_O = tmem_base + 128u;     // columns [128,256)
 
   if (warp == 4) {
-    // ------------------------------------------------------------------ issue warp (one lane)
+    // ------------------------------------------------------------------ MMA issue warp (one lane)
+    // Never waits for an MMA to finish: completion is signalled to the consumers of the result
+    // (S_FULL, O_DONE) and to the producer of the operands (K_FREE, V_FREE) through tcgen05.commit.
     if (lane == 0) {
       bool ok = true;
       const uint32_t idesc_qk = make_idesc(kTileN, false);
       const uint32_t idesc_pv = make_idesc(kD, true);
-      const int oob_row = p.num_pages * p.Hkv * kPage;      // a row coordinate past the end: zero fill
-
-      auto page_row = [&](int key0) -> int {
-        const int lp = key0 / kPage;
-        int pp = -1;
-        if (lp < p.max_pages) pp = p.block_table[(size_t)b * p.max_pages + lp];
-        if (pp < 0 || pp >= p.num_pages) {
-          if (key0 < kv_end && p.status) atomicOr(p.status, lp < p.max_pages ? WEDLM_STATUS_BAD_PAGE : WEDLM_STATUS_BAD_LENGTH);
-          return oob_row;
-        }
-        return (pp * p.Hkv + g) * kPage;
-      };
-      auto load_tile = [&](const CUtensorMap* map, uint32_t dst_stage, uint32_t full_bar, int t) {
-        mbar_expect_tx(full_bar, kStageBytes);
-#pragma unroll
-        for (int pg = 0; pg < kPagesPerTile; ++pg) {
-          const int y = page_row(kv_begin + t * kTileN + pg * kPage);
-          tma_load_2d(dst_stage + pg * 2048u, map, 0, y, full_bar);
-          tma_load_2d(dst_stage + kHalfKV + pg * 2048u, map, 64, y, full_bar);
-        }
-      };
-
-      // Q tile: two 64-element halves of [W_t slots x G heads] rows
-      const int q_slots = min(p.W_t, p.W);        // box height along the window dimension
-      mbar_expect_tx(bar(Q_FULL), (uint32_t)(2 * 64 * p.G * q_slots * 2));
-      tma_load_4d(sbase + kOffQ, &tm_q, 0, g * p.G, slot0, b, bar(Q_FULL));
-      tma_load_4d(sbase + kOffQ + kHalfQ, &tm_q, 64, g * p.G, slot0, b, bar(Q_FULL));
-      for (int t = 0; t < 2 && t < T; ++t) {
-        load_tile(&tm_k, sbase + kOffK + t * kStageBytes, bar(K_FULL0 + t), t);
-        load_tile(&tm_v, sbase + kOffV + t * kStageBytes, bar(V_FULL0 + t), t);
-      }
       auto issue_qk = [&](int t) {
         const uint32_t st = (uint32_t)t & 1u;
         tc_fence_after();
@@ -273,8 +245,8 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           umma(tmem_S + st * 64u, ad, bd, idesc_qk, kk > 0);
         }
         umma_commit(bar(S_FULL0 + st));
+        umma_commit(bar(K_FREE0 + st));
       };
-
       ok = mbar_wait(bar(Q_FULL), 0);
       if (ok) ok = mbar_wait(bar(K_FULL0), 0);
       if (ok) issue_qk(0);
@@ -282,16 +254,9 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t st = (uint32_t)t & 1u, ph = ((uint32_t)t >> 1) & 1u;
         if (t + 1 < T) {
           // S[(t+1)&1] was last read by the softmax of tile t-1, whose P_READY we saw one iteration ago
-          const uint32_t st1 = st ^ 1u, ph1 = ((uint32_t)(t + 1) >> 1) & 1u;
-          ok = mbar_wait(bar(K_FULL0 + st1), ph1);
+          ok = mbar_wait(bar(K_FULL0 + (st ^ 1u)), ((uint32_t)(t + 1) >> 1) & 1u);
           if (!ok) break;
           issue_qk(t + 1);
-        }
-        if (t + 2 < T) {
-          // K stage st is free once Q K_t^T has completed
-          ok = mbar_wait(bar(S_FULL0 + st), ph);
-          if (!ok) break;
-          load_tile(&tm_k, sbase + kOffK + st * kStageBytes, bar(K_FULL0 + st), t + 2);
         }
         ok = mbar_wait(bar(P_READY), (uint32_t)t & 1u);
         if (!ok) break;
@@ -305,12 +270,66 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           umma(tmem_O, ad, bd, idesc_pv, (t > 0) || (j > 0));
         }
         umma_commit(bar(O_DONE));
-        if (t + 2 < T) {
-          // V stage st is free once P V_t has completed
-          ok = mbar_wait(bar(O_DONE), (uint32_t)t & 1u);
-          if (!ok) break;
-          load_tile(&tm_v, sbase + kOffV + st * kStageBytes, bar(V_FULL0 + st), t + 2);
+        umma_commit(bar(V_FREE0 + st));
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        if (p.status) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ TMA producer warp (one lane)
+    if (lane == 0) {
+      bool ok = true;
+      const int oob_row = p.num_pages * p.Hkv * kPage;      // a row coordinate past the end: zero fill
+      // TMA row coordinate of the page that holds key0 (same for K and V)
+      auto page_row = [&](int key0) -> int {
+        const int lp = key0 / kPage;
+        int pp = -1;
+        if (lp < p.max_pages) pp = p.block_table[(size_t)b * p.max_pages + lp];
+        if (pp < 0 || pp >= p.num_pages) {
+          if (key0 < kv_end && p.status) atomicOr(p.status, lp < p.max_pages ? WEDLM_STATUS_BAD_PAGE : WEDLM_STATUS_BAD_LENGTH);
+          return oob_row;
         }
+        return (pp * p.Hkv + g) * kPage;
+      };
+      // page rows of the tiles in flight: a 4-tile ring in shared memory, written and read by this lane
+      volatile int* ring = reinterpret_cast<volatile int*>(smem + kOffBar + 128);
+      auto fetch_rows = [&](int t) {
+#pragma unroll
+        for (int pg = 0; pg < kPagesPerTile; ++pg)
+          ring[(t & 3) * kPagesPerTile + pg] = page_row(kv_begin + t * kTileN + pg * kPage);
+      };
+      auto load_tile = [&](const CUtensorMap* map, uint32_t dst_stage, uint32_t full_bar, int t) {
+        mbar_expect_tx(full_bar, kStageBytes);
+#pragma unroll
+        for (int pg = 0; pg < kPagesPerTile; ++pg) {
+          const int y = ring[(t & 3) * kPagesPerTile + pg];
+          tma_load_2d(dst_stage + pg * 2048u, map, 0, y, full_bar);
+          tma_load_2d(dst_stage + kHalfKV + pg * 2048u, map, 64, y, full_bar);
+        }
+      };
+      // Q tile: two 64-element halves of [W_t slots x G heads] rows
+      const int q_slots = min(p.W_t, p.W);        // box height along the window dimension
+      mbar_expect_tx(bar(Q_FULL), (uint32_t)(2 * 64 * p.G * q_slots * 2));
+      tma_load_4d(sbase + kOffQ, &tm_q, 0, g * p.G, slot0, b, bar(Q_FULL));
+      tma_load_4d(sbase + kOffQ + kHalfQ, &tm_q, 64, g * p.G, slot0, b, bar(Q_FULL));
+      // order of issue follows the order in which stages come free: K_{u+1} (after Q K_{u-1}^T), then
+      // V_u (after P V_{u-2})
+      fetch_rows(0);
+      load_tile(&tm_k, sbase + kOffK, bar(K_FULL0), 0);
+      for (int u = 0; ok && u < T; ++u) {
+        if (u + 1 < T) {
+          const uint32_t st1 = (uint32_t)(u + 1) & 1u;
+          fetch_rows(u + 1);
+          if (u + 1 >= 2) ok = mbar_wait(bar(K_FREE0 + st1), ((uint32_t)(u - 1) >> 1) & 1u);
+          if (!ok) break;
+          load_tile(&tm_k, sbase + kOffK + st1 * kStageBytes, bar(K_FULL0 + st1), u + 1);
+        }
+        const uint32_t st = (uint32_t)u & 1u;
+        if (u >= 2) ok = mbar_wait(bar(V_FREE0 + st), ((uint32_t)(u - 2) >> 1) & 1u);
+        if (!ok) break;
+        load_tile(&tm_v, sbase + kOffV + st * kStageBytes, bar(V_FULL0 + st), u);
       }
       if (!ok) {
         *abort_flag = 1;
