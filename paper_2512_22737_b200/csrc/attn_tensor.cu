@@ -28,7 +28,7 @@ namespace {
 constexpr int kTileN = 64;            // keys per tile (4 pages)
 constexpr int kD = 128;               // head size
 constexpr int kPage = 16;
-constexpr int kPagesPerTile = kTileN / kPage;
+static_assert(kTileN == 4 * kPage, "a tile is four pages");
 constexpr int kThreadsT = 192;        // 4 softmax warps + MMA issue warp + TMA producer warp
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kLazyRescaleLog2 = 8.0f;   // keep the old reference while the max grew by < 2^8
@@ -44,6 +44,7 @@ constexpr uint32_t kStageBytes = 16384;
 constexpr uint32_t kHalfKV = 8192;
 constexpr uint32_t kHalfQ = 16384;
 
+// (the TRACE macro below is empty in normal builds)
 enum Bar { Q_FULL = 0, K_FULL0, K_FULL1, V_FULL0, V_FULL1, S_FULL0, S_FULL1, O_DONE, P_READY, K_FREE0, K_FREE1,
            V_FREE0, V_FREE1, N_BARS };
 
@@ -57,6 +58,14 @@ struct TensorAttnParams {
   float* part_ml;
   int32_t* status;
 };
+
+#ifdef WEDLM_ATTN_TRACE
+// Debug builds only: per-tile timestamps of one CTA, [role][tile][event].
+__device__ long long g_attn_trace[3 * 256 * 8];
+#define TRACE(role, t, ev) do { if (trace_on && (unsigned)(t) < 256u) g_attn_trace[((role) * 256 + (t)) * 8 + (ev)] = clock64(); } while (0)
+#else
+#define TRACE(role, t, ev) do { } while (0)
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -155,6 +164,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+__device__ __forceinline__ float ex2_approx(float x) {      // 2^x on the SFU; flushes tiny results to zero
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -186,6 +200,9 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const int h = g * p.G + r % p.G;                           // query head
   const bool row_valid = (tid < 128) && (i_row < p.W);
   const float c = p.scale_log2;
+#ifdef WEDLM_ATTN_TRACE
+  const bool trace_on = (blockIdx.x == 0 && blockIdx.y == 3 && blockIdx.z == 0) && (lane == 0);
+#endif
 
   if (T == 0) {
     // nothing visible in this chunk for these rows: an empty partial (only possible when n_splits > 1)
@@ -244,6 +261,7 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           const uint64_t bd = make_desc(sbase + kOffK + st * kStageBytes + (kk >> 2) * kHalfKV + (kk & 3) * 32u, 16u, 1024u);
           umma(tmem_S + st * 64u, ad, bd, idesc_qk, kk > 0);
         }
+        TRACE(0, t - 1, 6);
         umma_commit(bar(S_FULL0 + st));
         umma_commit(bar(K_FREE0 + st));
       };
@@ -254,14 +272,19 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t st = (uint32_t)t & 1u, ph = ((uint32_t)t >> 1) & 1u;
         if (t + 1 < T) {
           // S[(t+1)&1] was last read by the softmax of tile t-1, whose P_READY we saw one iteration ago
+          TRACE(0, t, 0);
           ok = mbar_wait(bar(K_FULL0 + (st ^ 1u)), ((uint32_t)(t + 1) >> 1) & 1u);
           if (!ok) break;
+          TRACE(0, t, 1);
           issue_qk(t + 1);
+          TRACE(0, t, 2);
         }
         ok = mbar_wait(bar(P_READY), (uint32_t)t & 1u);
         if (!ok) break;
+        TRACE(0, t, 3);
         ok = mbar_wait(bar(V_FULL0 + st), ph);
         if (!ok) break;
+        TRACE(0, t, 4);
         tc_fence_after();
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -271,6 +294,7 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         umma_commit(bar(O_DONE));
         umma_commit(bar(V_FREE0 + st));
+        TRACE(0, t, 5);
       }
       if (!ok) {
         *abort_flag = 1;
@@ -278,63 +302,69 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
     }
   } else if (warp == 5) {
-    // ------------------------------------------------------------------ TMA producer warp (one lane)
+    // ------------------------------------------------------------------ TMA producer warp
+    // A tile is 8 copies of 2 KB (4 pages x 2 column halves).  Lanes 0..7 each look up their page and
+    // issue their copy, so that the 8 copies of a tile leave in one warp instruction.
+    bool ok = true;
+    const int oob_row = p.num_pages * p.Hkv * kPage;        // a row coordinate past the end: zero fill
+    const int pg = (lane >> 1) & 3, half = lane & 1;
+    const uint32_t lane_dst = (uint32_t)pg * 2048u + (uint32_t)half * kHalfKV;
+    // TMA row coordinate of this lane's page of tile t (same for K and V)
+    auto page_row = [&](int t) -> int {
+      const int key0 = kv_begin + t * kTileN + pg * kPage;
+      const int lp = key0 / kPage;
+      int pp = -1;
+      if (lp < p.max_pages) pp = p.block_table[(size_t)b * p.max_pages + lp];
+      if (pp < 0 || pp >= p.num_pages) {
+        if (key0 < kv_end && p.status) atomicOr(p.status, lp < p.max_pages ? WEDLM_STATUS_BAD_PAGE : WEDLM_STATUS_BAD_LENGTH);
+        return oob_row;
+      }
+      return (pp * p.Hkv + g) * kPage;
+    };
+    auto load_tile = [&](const CUtensorMap* map, uint32_t dst_stage, uint32_t full_bar, int y) {
+      if (lane == 0) mbar_expect_tx(full_bar, kStageBytes);
+      __syncwarp();
+      if (lane < 8) tma_load_2d(dst_stage + lane_dst, map, half * 64, y, full_bar);
+    };
+    auto wait_all = [&](uint32_t barrier, uint32_t parity) -> bool {      // lane 0 waits, the warp follows
+      int good = 1;
+      if (lane == 0) good = mbar_wait(barrier, parity) ? 1 : 0;
+      return __shfl_sync(0xffffffffu, good, 0) != 0;
+    };
     if (lane == 0) {
-      bool ok = true;
-      const int oob_row = p.num_pages * p.Hkv * kPage;      // a row coordinate past the end: zero fill
-      // TMA row coordinate of the page that holds key0 (same for K and V)
-      auto page_row = [&](int key0) -> int {
-        const int lp = key0 / kPage;
-        int pp = -1;
-        if (lp < p.max_pages) pp = p.block_table[(size_t)b * p.max_pages + lp];
-        if (pp < 0 || pp >= p.num_pages) {
-          if (key0 < kv_end && p.status) atomicOr(p.status, lp < p.max_pages ? WEDLM_STATUS_BAD_PAGE : WEDLM_STATUS_BAD_LENGTH);
-          return oob_row;
-        }
-        return (pp * p.Hkv + g) * kPage;
-      };
-      // page rows of the tiles in flight: a 4-tile ring in shared memory, written and read by this lane
-      volatile int* ring = reinterpret_cast<volatile int*>(smem + kOffBar + 128);
-      auto fetch_rows = [&](int t) {
-#pragma unroll
-        for (int pg = 0; pg < kPagesPerTile; ++pg)
-          ring[(t & 3) * kPagesPerTile + pg] = page_row(kv_begin + t * kTileN + pg * kPage);
-      };
-      auto load_tile = [&](const CUtensorMap* map, uint32_t dst_stage, uint32_t full_bar, int t) {
-        mbar_expect_tx(full_bar, kStageBytes);
-#pragma unroll
-        for (int pg = 0; pg < kPagesPerTile; ++pg) {
-          const int y = ring[(t & 3) * kPagesPerTile + pg];
-          tma_load_2d(dst_stage + pg * 2048u, map, 0, y, full_bar);
-          tma_load_2d(dst_stage + kHalfKV + pg * 2048u, map, 64, y, full_bar);
-        }
-      };
       // Q tile: two 64-element halves of [W_t slots x G heads] rows
       const int q_slots = min(p.W_t, p.W);        // box height along the window dimension
       mbar_expect_tx(bar(Q_FULL), (uint32_t)(2 * 64 * p.G * q_slots * 2));
       tma_load_4d(sbase + kOffQ, &tm_q, 0, g * p.G, slot0, b, bar(Q_FULL));
       tma_load_4d(sbase + kOffQ + kHalfQ, &tm_q, 64, g * p.G, slot0, b, bar(Q_FULL));
-      // order of issue follows the order in which stages come free: K_{u+1} (after Q K_{u-1}^T), then
-      // V_u (after P V_{u-2})
-      fetch_rows(0);
-      load_tile(&tm_k, sbase + kOffK, bar(K_FULL0), 0);
-      for (int u = 0; ok && u < T; ++u) {
-        if (u + 1 < T) {
-          const uint32_t st1 = (uint32_t)(u + 1) & 1u;
-          fetch_rows(u + 1);
-          if (u + 1 >= 2) ok = mbar_wait(bar(K_FREE0 + st1), ((uint32_t)(u - 1) >> 1) & 1u);
-          if (!ok) break;
-          load_tile(&tm_k, sbase + kOffK + st1 * kStageBytes, bar(K_FULL0 + st1), u + 1);
-        }
-        const uint32_t st = (uint32_t)u & 1u;
-        if (u >= 2) ok = mbar_wait(bar(V_FREE0 + st), ((uint32_t)(u - 2) >> 1) & 1u);
+    }
+    // order of issue follows the order in which stages come free: K_{u+1} (after Q K_{u-1}^T), then
+    // V_u (after P V_{u-2})
+    int y_cur = page_row(0);
+    load_tile(&tm_k, sbase + kOffK, bar(K_FULL0), y_cur);
+    int y_next = (1 < T) ? page_row(1) : oob_row;
+    for (int u = 0; ok && u < T; ++u) {
+      if (u + 1 < T) {
+        const uint32_t st1 = (uint32_t)(u + 1) & 1u;
+        TRACE(1, u, 0);
+        if (u + 1 >= 2) ok = wait_all(bar(K_FREE0 + st1), ((uint32_t)(u - 1) >> 1) & 1u);
         if (!ok) break;
-        load_tile(&tm_v, sbase + kOffV + st * kStageBytes, bar(V_FULL0 + st), u);
+        TRACE(1, u, 2);
+        load_tile(&tm_k, sbase + kOffK + st1 * kStageBytes, bar(K_FULL0 + st1), y_next);
+        TRACE(1, u, 3);
       }
-      if (!ok) {
-        *abort_flag = 1;
-        if (p.status) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
-      }
+      const uint32_t st = (uint32_t)u & 1u;
+      if (u >= 2) ok = wait_all(bar(V_FREE0 + st), ((uint32_t)(u - 2) >> 1) & 1u);
+      if (!ok) break;
+      TRACE(1, u, 4);
+      load_tile(&tm_v, sbase + kOffV + st * kStageBytes, bar(V_FULL0 + st), y_cur);
+      TRACE(1, u, 5);
+      y_cur = y_next;
+      if (u + 2 < T) y_next = page_row(u + 2);      // consumed one iteration later
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      if (p.status) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
     }
   } else {
     // ------------------------------------------------------------------ softmax warps: one row per thread
@@ -345,8 +375,10 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     bool ok = true;
     for (int t = 0; t < T; ++t) {
       const uint32_t st = (uint32_t)t & 1u, ph = ((uint32_t)t >> 1) & 1u;
+      TRACE(2, t, 0);
       ok = mbar_wait(bar(S_FULL0 + st), ph);
       if (!ok) break;
+      TRACE(2, t, 1);
       tc_fence_after();
       uint32_t raw[64];
       {
@@ -356,6 +388,7 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tmem_ld32(tmem_S + lane_sel + st * 64u + 32u, hi);
         tmem_wait_ld();
       }
+      TRACE(2, t, 2);
       float s[64];
       const int tile0 = kv_begin + t * kTileN;
       const bool need_mask = tile0 + kTileN > min(P + slot0 + 1, kv_end);   // block-uniform
@@ -370,11 +403,17 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           m_tile = fmaxf(m_tile, x);
         }
       } else {
+        float m4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-        for (int cc = 0; cc < 64; ++cc) {
-          s[cc] = __uint_as_float(raw[cc]);
-          m_tile = fmaxf(m_tile, s[cc]);
+        for (int cc = 0; cc < 64; cc += 8) {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) s[cc + e] = __uint_as_float(raw[cc + e]);
+          m4[0] = fmaxf(m4[0], fmaxf(s[cc + 0], s[cc + 1]));
+          m4[1] = fmaxf(m4[1], fmaxf(s[cc + 2], s[cc + 3]));
+          m4[2] = fmaxf(m4[2], fmaxf(s[cc + 4], s[cc + 5]));
+          m4[3] = fmaxf(m4[3], fmaxf(s[cc + 6], s[cc + 7]));
         }
+        m_tile = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
       }
       // lazy reference: only move it when the maximum grew by more than 2^kLazyRescaleLog2
       float alpha = 1.f;
@@ -385,20 +424,22 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         moved = true;
       }
       const float neg_mc = (m_ref == -CUDART_INF_F) ? 0.f : -m_ref * c;
-      float sum = 0.f;
+      float sum = 0.f, sum2 = 0.f;
       uint32_t pk[32];
 #pragma unroll
       for (int cc = 0; cc < 64; cc += 2) {
-        const float p0 = exp2f(fmaf(s[cc], c, neg_mc));
-        const float p1 = exp2f(fmaf(s[cc + 1], c, neg_mc));
-        sum += p0 + p1;
+        const float p0 = ex2_approx(fmaf(s[cc], c, neg_mc));
+        const float p1 = ex2_approx(fmaf(s[cc + 1], c, neg_mc));
+        if ((cc & 2) == 0) sum += p0 + p1; else sum2 += p0 + p1;
         pk[cc >> 1] = pack_bf16(p0, p1);
       }
-      l = l * alpha + sum;
+      l = l * alpha + (sum + sum2);
       // P buffer and O are free / stable once P V_{t-1} has completed
+      TRACE(2, t, 3);
       if (t > 0) {
         ok = mbar_wait(bar(O_DONE), (uint32_t)(t - 1) & 1u);
         if (!ok) break;
+        TRACE(2, t, 4);
         tc_fence_after();
         if (__any_sync(0xffffffffu, moved)) {
 #pragma unroll 1
@@ -433,9 +474,11 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           *reinterpret_cast<uint4*>(vst + (ch >> 3) * kHalfKV + row * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
         }
       }
+      TRACE(2, t, 5);
       fence_async_smem();
       tc_fence_before();
       mbar_arrive(bar(P_READY));
+      TRACE(2, t, 6);
     }
     if (ok) ok = mbar_wait(bar(O_DONE), (uint32_t)(T - 1) & 1u);
     if (!ok) {
@@ -506,6 +549,12 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
 }
 
 }  // namespace
+
+#ifdef WEDLM_ATTN_TRACE
+extern "C" int wedlm_debug_read_attn_trace(long long* host_dst) {
+  return cudaMemcpyFromSymbol(host_dst, g_attn_trace, sizeof(long long) * 3 * 256 * 8) == cudaSuccess ? 0 : -4;
+}
+#endif
 
 bool attn_tensor_supported(const wedlm_config_t* c) {
   if (c->dtype != WEDLM_DTYPE_BF16 || c->head_dim != kD || c->page_size != kPage) return false;
