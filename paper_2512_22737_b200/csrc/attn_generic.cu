@@ -132,7 +132,7 @@ attn_generic_kernel(Shape s, int n_splits, int chunk, const T* __restrict__ q_ro
     const int rr = r * RSTRIDE + rofs;
     if (rr >= rows) continue;
     const size_t qrow = ((size_t)b * s.W + row0 + rr) * s.Hq + h;       // (b, i, h)
-    if (n_splits == 1) {
+    if (n_valid == 1) {
       const float inv = ls[rr] > 0.f ? 1.f / ls[rr] : 0.f;
 #pragma unroll
       for (int c = 0; c < CPT; ++c) st_from_float(out, qrow * D + col0 + c * kThreads, acc[r][c] * inv);
@@ -146,31 +146,43 @@ attn_generic_kernel(Shape s, int n_splits, int chunk, const T* __restrict__ q_ro
 }
 
 // Merge of split partials (m, l, o): m = max m_s; w_s = 2^(m_s - m); out = sum w_s o_s / sum w_s l_s.
-// grid (W, Hq, B), D threads (or fewer, looping).  Partials hold m in the log2 domain.
+// One warp per (b, i, h) output row; lanes stride over D with 16-byte loads.  Sequences whose keys fit
+// one chunk were written directly by the attention kernel and are skipped.  m is in the log2 domain.
 template <typename T>
-__global__ void attn_merge_kernel(Shape s, int n_splits, int chunk, const int32_t* __restrict__ prefix_len,
-                                  const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                  T* __restrict__ out) {
-  const int i = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+__global__ void __launch_bounds__(256)
+attn_merge_kernel(Shape s, int n_splits, int chunk, const int32_t* __restrict__ prefix_len,
+                  const float* __restrict__ part_o, const float* __restrict__ part_ml, T* __restrict__ out) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  const int rows_per_seq = s.Hq * s.W;
+  if (warp >= s.B * rows_per_seq) return;
+  const int b = warp / rows_per_seq, rem = warp - b * rows_per_seq;
+  const int h = rem / s.W, i = rem - h * s.W;                       // partial rows are ordered (b, h, i)
   const int P = max(prefix_len[b], 0);
   const int n_valid = min(n_splits, (P + s.W + chunk - 1) / chunk);
-  const size_t prow = (((size_t)b * s.Hq + h) * s.W + i) * n_splits;
+  if (n_valid <= 1) return;
+  const size_t prow = (size_t)warp * n_splits;
   float m = -CUDART_INF_F;
   for (int sp = 0; sp < n_valid; ++sp) m = fmaxf(m, part_ml[(prow + sp) * 2]);
   float l = 0.f;
   for (int sp = 0; sp < n_valid; ++sp) {
-    float ms = part_ml[(prow + sp) * 2];
+    const float ms = part_ml[(prow + sp) * 2];
     if (ms != -CUDART_INF_F) l += exp2f(ms - m) * part_ml[(prow + sp) * 2 + 1];
   }
   const float inv = l > 0.f ? 1.f / l : 0.f;
   const size_t orow = (((size_t)b * s.W + i) * s.Hq + h) * s.D;
-  for (int d = threadIdx.x; d < s.D; d += blockDim.x) {
-    float o = 0.f;
+  for (int d = lane * 4; d < s.D; d += 128) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int sp = 0; sp < n_valid; ++sp) {
-      float ms = part_ml[(prow + sp) * 2];
-      if (ms != -CUDART_INF_F) o += exp2f(ms - m) * part_o[(prow + sp) * s.D + d];
+      const float ms = part_ml[(prow + sp) * 2];
+      if (ms == -CUDART_INF_F) continue;
+      const float w = exp2f(ms - m);
+      const float4 o = *reinterpret_cast<const float4*>(part_o + (prow + sp) * s.D + d);
+      acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
     }
-    st_from_float(out, orow + d, o * inv);
+    st_from_float(out, orow + d, acc.x * inv);
+    st_from_float(out, orow + d + 1, acc.y * inv);
+    st_from_float(out, orow + d + 2, acc.z * inv);
+    st_from_float(out, orow + d + 3, acc.w * inv);
   }
 }
 
@@ -216,12 +228,12 @@ int launch_attn_generic(const Shape& s, const AttnPlan& plan, const void* q_rot,
 
 int launch_attn_merge(const Shape& s, const AttnPlan& plan, const int32_t* prefix_len, const float* part_o,
                       const float* part_ml, void* out, cudaStream_t st) {
-  dim3 grid(s.W, s.Hq, s.B);
-  int threads = s.D < 128 ? s.D : 128;
+  const long long warps = (long long)s.B * s.Hq * s.W;
+  const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
   if (s.dtype == WEDLM_DTYPE_BF16)
-    attn_merge_kernel<__nv_bfloat16><<<grid, threads, 0, st>>>(s, plan.n_splits, plan.chunk, prefix_len, part_o, part_ml, (__nv_bfloat16*)out);
+    attn_merge_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(s, plan.n_splits, plan.chunk, prefix_len, part_o, part_ml, (__nv_bfloat16*)out);
   else
-    attn_merge_kernel<float><<<grid, threads, 0, st>>>(s, plan.n_splits, plan.chunk, prefix_len, part_o, part_ml, (float*)out);
+    attn_merge_kernel<float><<<blocks, 256, 0, st>>>(s, plan.n_splits, plan.chunk, prefix_len, part_o, part_ml, (float*)out);
   count_launch();
   return cuda_ok(cudaGetLastError());
 }

@@ -206,7 +206,7 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   if (T == 0) {
     // nothing visible in this chunk for these rows: an empty partial (only possible when n_splits > 1)
-    if (row_valid && p.n_splits > 1) {
+    if (row_valid && n_valid > 1) {
       const size_t prow = (((size_t)b * p.Hq + h) * p.W + i_row) * p.n_splits + split;
       float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
       float4* dst = reinterpret_cast<float4*>(p.part_o + prow * kD);
@@ -486,7 +486,7 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       if (p.status) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
     } else {
       tc_fence_after();
-      const bool final_out = p.n_splits == 1;
+      const bool final_out = n_valid == 1;        // the only chunk of this sequence: write the result itself
       const float inv = l > 0.f ? 1.f / l : 0.f;
       const size_t orow = (((size_t)b * p.W + i_row) * p.Hq + h) * kD;
       const size_t prow = (((size_t)b * p.Hq + h) * p.W + i_row) * p.n_splits + split;

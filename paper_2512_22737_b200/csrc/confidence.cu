@@ -80,44 +80,62 @@ conf_partial_kernel(int W, int V, int n_chunks, const T* __restrict__ logits, co
         x[k * VL + e] = idx < V ? ld_as_float(src, idx) : -CUDART_INF_F;
       }
   }
-  // thread-local arg-max in increasing index order (strict > keeps the lowest index)
-  float m = -CUDART_INF_F;
-  int a = 0x7fffffff;
+  // chunk maximum: values only (tree for ILP), then one shuffle reduction and one shared-memory hop
+  float mt[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-  for (int k = 0; k < kConfVecs; ++k)
-#pragma unroll
-    for (int e = 0; e < VL; ++e) {
-      int idx = base + (k * kConfThreads + tid) * VL + e;
-      if (x[k * VL + e] > m) { m = x[k * VL + e]; a = idx; }
-    }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    float ov = __shfl_xor_sync(0xffffffffu, m, o);
-    int oi = __shfl_xor_sync(0xffffffffu, a, o);
-    argmax_combine(m, a, ov, oi);
+  for (int k = 0; k < EPT; k += 4) {
+    mt[0] = fmaxf(mt[0], x[k]);
+    mt[1] = fmaxf(mt[1], x[k + 1]);
+    mt[2] = fmaxf(mt[2], x[k + 2]);
+    mt[3] = fmaxf(mt[3], x[k + 3]);
   }
+  const float m_thread = fmaxf(fmaxf(mt[0], mt[1]), fmaxf(mt[2], mt[3]));
+  float m = m_thread;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
   __shared__ float sm_m[kConfThreads / 32];
-  __shared__ int sm_a[kConfThreads / 32];
   __shared__ float sm_s[kConfThreads / 32];
   __shared__ float sm_t[kConfThreads / 32];
+  __shared__ int sm_a;
   const int warp = tid >> 5, lane = tid & 31;
-  if (lane == 0) { sm_m[warp] = m; sm_a[warp] = a; }
+  if (lane == 0) sm_m[warp] = m;
+  if (tid == 0) sm_a = 0x7fffffff;
   __syncthreads();
-  m = sm_m[0]; a = sm_a[0];
+  m = sm_m[0];
 #pragma unroll
-  for (int w = 1; w < kConfThreads / 32; ++w) argmax_combine(m, a, sm_m[w], sm_a[w]);
+  for (int w = 1; w < kConfThreads / 32; ++w) m = fmaxf(m, sm_m[w]);
+  // lowest index attaining the maximum: only the few threads that hold it look for it
+  if (m_thread == m) {
+    int a = 0x7fffffff;
+#pragma unroll
+    for (int k = kConfVecs - 1; k >= 0; --k)
+#pragma unroll
+      for (int e = VL - 1; e >= 0; --e)
+        if (x[k * VL + e] == m) a = base + (k * kConfThreads + tid) * VL + e;     // descending scan keeps the lowest
+    atomicMin(&sm_a, a);
+  }
 
-  // sums relative to the chunk maximum; terms whose exponential underflows to 0 add 0
-  float s = 0.f, t = 0.f;
+  // sums relative to the chunk maximum in the log2 domain: d = (x - m) log2(e), e = 2^d,
+  // s = sum e, t = ln2 * sum d e.  d is clamped at -127, where e has already flushed to zero, so that
+  // -inf logits (and the padding) add exactly 0 instead of inf * 0.
+  float s0 = 0.f, s1 = 0.f, t0 = 0.f, t1 = 0.f;
   if (m > -CUDART_INF_F) {
+    const float kLog2e = 1.4426950408889634f;
+    const float nm = -m * kLog2e;
 #pragma unroll
-    for (int k = 0; k < EPT; ++k) {
-      float d = x[k] - m;
-      float e = exp2f(d * 1.4426950408889634f);
-      s += e;
-      t += (e > 0.f) ? d * e : 0.f;
+    for (int k = 0; k < EPT; k += 2) {
+      const float d0 = fmaxf(fmaf(x[k], kLog2e, nm), -127.f);
+      const float d1 = fmaxf(fmaf(x[k + 1], kLog2e, nm), -127.f);
+      float e0, e1;
+      asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(d0));
+      asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(d1));
+      s0 += e0;
+      s1 += e1;
+      t0 = fmaf(d0, e0, t0);
+      t1 = fmaf(d1, e1, t1);
     }
   }
+  float s = s0 + s1, t = (t0 + t1) * 0.6931471805599453f;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     s += __shfl_xor_sync(0xffffffffu, s, o);
@@ -129,7 +147,7 @@ conf_partial_kernel(int W, int V, int n_chunks, const T* __restrict__ logits, co
     float ss = 0.f, tt = 0.f;
 #pragma unroll
     for (int w = 0; w < kConfThreads / 32; ++w) { ss += sm_s[w]; tt += sm_t[w]; }
-    part[(size_t)row * n_chunks + chunk] = make_float4(m, ss, tt, __int_as_float(a));
+    part[(size_t)row * n_chunks + chunk] = make_float4(m, ss, tt, __int_as_float(sm_a));
   }
 }
 

@@ -1,15 +1,20 @@
 // RoPE at the supplied logical position ids (Section 2.2) for the window's q and k, and staging
 // of the rotated k and of v into the paged cache at positions prefix_len + i ("Extend (K, V)" of
 // Algorithm 1, done for every physical row so that a commit is just prefix_len += n).
+#include <cmath>
+
 #include "common.cuh"
 
 namespace wedlm {
+
+// theta^(-2d/D) for d < D/2, computed on the host in double and passed by value (D <= 256).
+struct InvFreq { double v[128]; };
 
 // grid (W, B); one block per (physical row i, sequence b).  Angles are formed in double so that
 // positions of tens of thousands keep full fp32 accuracy after the range reduction.
 template <typename T>
 __global__ void __launch_bounds__(128)
-rope_stage_kernel(Shape s, const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+rope_stage_kernel(Shape s, const InvFreq inv_freq, const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                   T* __restrict__ q_rot, T* __restrict__ k_cache, T* __restrict__ v_cache,
                   const int32_t* __restrict__ block_table, const int32_t* __restrict__ prefix_len,
                   const int32_t* __restrict__ pos_ids, const int32_t* __restrict__ count,
@@ -23,11 +28,14 @@ rope_stage_kernel(Shape s, const T* __restrict__ q, const T* __restrict__ k, con
   if (rotate) {
     const double pos = (double)pos_ids[(size_t)b * s.W + i];
     for (int d = tid; d < half; d += blockDim.x) {
-      double inv_freq = pow((double)s.theta, -2.0 * (double)d / (double)D);
-      double sv, cv;
-      sincos(pos * inv_freq, &sv, &cv);
-      cs[d] = (float)cv;
-      sn[d] = (float)sv;
+      // the angle is formed and reduced to [-pi, pi] in double (positions reach tens of thousands of
+      // radians), the sine and cosine of the reduced angle are then accurate in fp32
+      const double ang = pos * inv_freq.v[d];
+      const double red = ang - 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
+      float sv, cv;
+      sincosf((float)red, &sv, &cv);
+      cs[d] = cv;
+      sn[d] = sv;
     }
   } else {
     for (int d = tid; d < half; d += blockDim.x) { cs[d] = 1.f; sn[d] = 0.f; }
@@ -75,14 +83,17 @@ int launch_rope_stage(const Shape& s, const void* q, const void* k, const void* 
                       const int32_t* count, int32_t* kv_slot_idx, int32_t* status, cudaStream_t st) {
   dim3 grid(s.W, s.B);
   size_t smem = (size_t)s.D * sizeof(float);
+  InvFreq inv_freq;
+  for (int d = 0; d < s.D / 2; ++d) inv_freq.v[d] = pow((double)s.theta, -2.0 * (double)d / (double)s.D);
+  for (int d = s.D / 2; d < 128; ++d) inv_freq.v[d] = 0.0;
   if (s.dtype == WEDLM_DTYPE_BF16) {
     using T = __nv_bfloat16;
-    rope_stage_kernel<T><<<grid, 128, smem, st>>>(s, (const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_cache,
+    rope_stage_kernel<T><<<grid, 128, smem, st>>>(s, inv_freq, (const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_cache,
                                                   (T*)v_cache, block_table, prefix_len, pos_ids, count, kv_slot_idx,
                                                   status);
   } else {
     using T = float;
-    rope_stage_kernel<T><<<grid, 128, smem, st>>>(s, (const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_cache,
+    rope_stage_kernel<T><<<grid, 128, smem, st>>>(s, inv_freq, (const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_cache,
                                                   (T*)v_cache, block_table, prefix_len, pos_ids, count, kv_slot_idx,
                                                   status);
   }
