@@ -34,6 +34,35 @@ __device__ __forceinline__ void unpack16(const uint4& u, float (&x)[4]) {
   x[0] = __uint_as_float(u.x); x[1] = __uint_as_float(u.y); x[2] = __uint_as_float(u.z); x[3] = __uint_as_float(u.w);
 }
 
+// Packed fp32x2 arithmetic of sm_100 (two lanes per instruction).
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float ex2_ftz(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t bf162_max(uint32_t a, uint32_t b) {
+  __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
+  return *reinterpret_cast<uint32_t*>(&r);
+}
+
 // (value, index) arg-max combine: larger value wins, equal values keep the lower index.
 __device__ __forceinline__ void argmax_combine(float& v, int& i, float ov, int oi) {
   if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
@@ -148,6 +177,194 @@ conf_partial_kernel(int W, int V, int n_chunks, const T* __restrict__ logits, co
 #pragma unroll
     for (int w = 0; w < kConfThreads / 32; ++w) { ss += sm_s[w]; tt += sm_t[w]; }
     part[(size_t)row * n_chunks + chunk] = make_float4(m, ss, tt, __int_as_float(sm_a));
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Streaming variant of pass 1 for bf16 logits with 16-byte aligned rows: persistent blocks pull
+// (row, chunk) items of active mask rows through a 4-stage shared-memory ring filled by bulk
+// asynchronous copies (one 16 KB copy per item, completion on an mbarrier), so that the bytes in
+// flight per SM do not depend on registers.  Same chunking and partial layout as conf_partial_kernel.
+// ------------------------------------------------------------------------------------------------
+constexpr int kStreamStages = 4;
+constexpr int kStreamChunk = kConfThreads * kConfVecs * 8;          // 8192 bf16 = 16 KB
+constexpr uint32_t kStreamSpin = 1u << 22;
+
+__device__ __forceinline__ uint32_t cs_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool cs_mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kStreamSpin; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+__device__ __forceinline__ void cs_consumer_sync() {     // the 256 consumer threads only
+  asm volatile("bar.sync 1, 256;" ::: "memory");
+}
+
+// block = 8 consumer warps (threads 0..255) + 1 producer warp (lane 0 of warp 8 issues the copies)
+__global__ void __launch_bounds__(kConfThreads + 32)
+conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv_bfloat16* __restrict__ logits,
+                   const int32_t* __restrict__ n_filled, const int32_t* __restrict__ window_len,
+                   float4* __restrict__ part) {
+  extern __shared__ __align__(128) unsigned char cs_smem[];
+  unsigned char* stage_mem = cs_smem;                                       // kStreamStages x 16 KB
+  uint64_t* full = reinterpret_cast<uint64_t*>(cs_smem + kStreamStages * kStreamChunk * 2);
+  uint64_t* empty = full + kStreamStages;
+  volatile long long* item_of = reinterpret_cast<volatile long long*>(empty + kStreamStages);
+  __shared__ float fm[kConfThreads / 32];
+  __shared__ float fs[kConfThreads / 32];
+  __shared__ float ft[kConfThreads / 32];
+  __shared__ int fa;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  long long cursor = blockIdx.x;                     // next candidate item of this block (producer only)
+
+  // producer: put the next active item of this block into stage st, or -1 when the block is done;
+  // returns false after the end marker
+  auto produce = [&](int st) -> bool {
+    const uint32_t bar = cs_smem_u32(full + st);
+    for (;;) {
+      const long long it = cursor;
+      cursor += gridDim.x;
+      if (it >= total_items) {
+        item_of[st] = -1;
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+        return false;
+      }
+      const int row = (int)(it / n_chunks), chunk = (int)(it - (long long)row * n_chunks);
+      const int b = row / W, i = row - b * W;
+      const int L = window_len ? min(max(window_len[b], 0), W) : W;
+      if (i < n_filled[b] || i >= L) continue;       // not an active mask row
+      const int base = chunk * kStreamChunk;
+      const uint32_t bytes = (uint32_t)min(kStreamChunk, V - base) * 2u;
+      item_of[st] = it;
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+      asm volatile(
+          "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+          ::"r"(cs_smem_u32(stage_mem + (size_t)st * kStreamChunk * 2)), "l"(logits + (size_t)row * V + base), "r"(bytes), "r"(bar)
+          : "memory");
+      return true;
+    }
+  };
+
+  if (tid == 0) {
+    for (int st = 0; st < kStreamStages; ++st) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(cs_smem_u32(full + st)));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(cs_smem_u32(empty + st)));
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == kConfThreads / 32) {
+    // ---- producer warp: fill the ring, then refill each stage as soon as the consumers release it
+    if (lane == 0) {
+      bool more = true;
+      for (uint32_t n = 0; more; ++n) {
+        const int st = n & (kStreamStages - 1);
+        if (n >= kStreamStages && !cs_mbar_wait(cs_smem_u32(empty + st), ((n / kStreamStages) - 1) & 1u)) break;
+        more = produce(st);
+      }
+    }
+    return;
+  }
+
+  for (uint32_t n = 0;; ++n) {
+    const int st = n & (kStreamStages - 1);
+    if (!cs_mbar_wait(cs_smem_u32(full + st), (n / kStreamStages) & 1u)) return;   // bounded; never expected
+    const long long it = item_of[st];
+    if (it < 0) break;
+    const int row = (int)(it / n_chunks), chunk = (int)(it - (long long)row * n_chunks);
+    const int base = chunk * kStreamChunk;
+    const uint4* src = reinterpret_cast<const uint4*>(stage_mem + (size_t)st * kStreamChunk * 2);
+    uint32_t w[kConfVecs * 4];
+#pragma unroll
+    for (int k = 0; k < kConfVecs; ++k) {
+      const uint4 v = src[k * kConfThreads + tid];
+      w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
+    }
+    if (base + kStreamChunk > V) {                   // last chunk of a row: words past the row end act as padding
+#pragma unroll
+      for (int i = 0; i < kConfVecs * 4; ++i) {
+        const int e0 = base + ((i >> 2) * kConfThreads + tid) * 8 + (i & 3) * 2;
+        if (e0 >= V) w[i] = 0xF149F149u;
+      }
+    }
+    // -inf logits are pulled up to -1e30 (bf16 pair 0xF149F149) so that they add exactly 0 below
+    uint32_t mx[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      w[q] = bf162_max(w[q], 0xF149F149u);
+      mx[q] = w[q];
+    }
+#pragma unroll
+    for (int i = 4; i < kConfVecs * 4; ++i) {
+      w[i] = bf162_max(w[i], 0xF149F149u);
+      mx[i & 3] = bf162_max(mx[i & 3], w[i]);
+    }
+    const uint32_t m2 = bf162_max(bf162_max(mx[0], mx[1]), bf162_max(mx[2], mx[3]));
+    const float m_thread = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xffff0000u));
+    float m = m_thread;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) fm[warp] = m;
+    if (tid == 0) fa = 0x7fffffff;
+    cs_consumer_sync();                              // also: every consumer holds its part of stage st in registers
+    if (tid == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(cs_smem_u32(empty + st)) : "memory");
+    m = fm[0];
+#pragma unroll
+    for (int q = 1; q < kConfThreads / 32; ++q) m = fmaxf(m, fm[q]);
+    if (m_thread == m) {                             // lowest index attaining the maximum (descending scan)
+      int a = 0x7fffffff;
+#pragma unroll
+      for (int i = kConfVecs * 4 - 1; i >= 0; --i) {
+        const int e0 = base + ((i >> 2) * kConfThreads + tid) * 8 + (i & 3) * 2;
+        if (__uint_as_float(w[i] & 0xffff0000u) == m) a = e0 + 1;
+        if (__uint_as_float(w[i] << 16) == m) a = e0;
+      }
+      atomicMin(&fa, a);
+    }
+    // d = (x - m) log2(e), e = 2^d, s = sum e, t = ln2 * sum d e, two logits per instruction
+    const float kLog2e = 1.4426950408889634f;
+    const unsigned long long L2 = pack2(kLog2e, kLog2e), NM = pack2(-m * kLog2e, -m * kLog2e);
+    unsigned long long sA = pack2(0.f, 0.f), sB = sA, tA = sA, tB = sA;
+#pragma unroll
+    for (int i = 0; i < kConfVecs * 4; i += 2) {
+      const unsigned long long dA = fma2(pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u)), L2, NM);
+      const unsigned long long dB = fma2(pack2(__uint_as_float(w[i + 1] << 16), __uint_as_float(w[i + 1] & 0xffff0000u)), L2, NM);
+      float a0, a1, b0, b1;
+      unpack2(dA, a0, a1);
+      unpack2(dB, b0, b1);
+      const unsigned long long eA = pack2(ex2_ftz(a0), ex2_ftz(a1));
+      const unsigned long long eB = pack2(ex2_ftz(b0), ex2_ftz(b1));
+      sA = add2(sA, eA);
+      sB = add2(sB, eB);
+      tA = fma2(dA, eA, tA);
+      tB = fma2(dB, eB, tB);
+    }
+    float s0, s1, t0, t1;
+    unpack2(add2(sA, sB), s0, s1);
+    unpack2(add2(tA, tB), t0, t1);
+    float ssum = s0 + s1, tsum = (t0 + t1) * 0.6931471805599453f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      ssum += __shfl_xor_sync(0xffffffffu, ssum, o);
+      tsum += __shfl_xor_sync(0xffffffffu, tsum, o);
+    }
+    if (lane == 0) { fs[warp] = ssum; ft[warp] = tsum; }
+    cs_consumer_sync();
+    if (tid == 0) {
+      float ss = 0.f, tt = 0.f;
+#pragma unroll
+      for (int q = 0; q < kConfThreads / 32; ++q) { ss += fs[q]; tt += ft[q]; }
+      part[(size_t)row * n_chunks + chunk] = make_float4(m, ss, tt, __int_as_float(fa));
+    }
   }
 }
 
@@ -334,8 +551,19 @@ int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* log
   if (s.dtype == WEDLM_DTYPE_BF16) {
     using T = __nv_bfloat16;
     const bool vec = (s.V % VecTraits<T>::VL == 0) && ((uintptr_t)logits % 16 == 0);
-    if (vec) conf_partial_kernel<T, true><<<(unsigned)blocks, kConfThreads, 0, st>>>(s.W, s.V, n_chunks, (const T*)logits, n_filled, window_len, part);
-    else     conf_partial_kernel<T, false><<<(unsigned)blocks, kConfThreads, 0, st>>>(s.W, s.V, n_chunks, (const T*)logits, n_filled, window_len, part);
+    if (vec) {
+      const size_t smem = (size_t)kStreamStages * kStreamChunk * 2 + kStreamStages * 24;
+      if (cudaFuncSetAttribute(conf_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return WEDLM_ERR_CUDA;
+      int dev = 0, sms = 148;
+      if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+      long long grid = (long long)sms * 3;                       // three 64 KB rings per SM
+      if (grid > blocks) grid = blocks;
+      conf_stream_kernel<<<(unsigned)grid, kConfThreads + 32, smem, st>>>(s.W, s.V, n_chunks, blocks, (const T*)logits, n_filled,
+                                                                      window_len, part);
+    } else {
+      conf_partial_kernel<T, false><<<(unsigned)blocks, kConfThreads, 0, st>>>(s.W, s.V, n_chunks, (const T*)logits, n_filled, window_len, part);
+    }
   } else {
     using T = float;
     const bool vec = (s.V % VecTraits<T>::VL == 0) && ((uintptr_t)logits % 16 == 0);
