@@ -75,10 +75,25 @@ AttnPlan plan_attention(const wedlm_config_t* c) {
     const int G = c->n_q_heads / c->n_kv_heads;
     const long long w_t = 128 / G;
     const long long units = (long long)c->batch * c->n_kv_heads * ((c->window + w_t - 1) / w_t);
-    long long want = units > 0 ? (3LL * 296 + units - 1) / units : 1;
-    if (const char* e = getenv("WEDLM_ATTN_SPLITS")) { long long v = atoll(e); if (v > 0) want = v; }
-    long long cap = total / 1024 > 1 ? total / 1024 : 1;                    // keep chunks >= 1024 keys
-    S = want < 1 ? 1 : (want > cap ? cap : want);
+    // Sequences are dispatched longest first, so a batch with at least one work unit per CTA slot
+    // (2 per SM) balances well without splitting the keys, and then no partials exist at all.  With
+    // fewer units the keys are split just far enough to fill the slots: the smallest split count
+    // whose last wave is at least 85 % full, chunks no shorter than 256 keys.
+    const long long slots = 2LL * 148;
+    long long cap = total / 256 > 1 ? total / 256 : 1;
+    if (cap > 64) cap = 64;
+    S = 1;
+    if (units > 0 && units < slots) {
+      double best = 0.0;
+      for (long long cand = 1; cand <= cap; ++cand) {
+        const long long ctas = units * cand;
+        const long long waves = (ctas + slots - 1) / slots;
+        const double eff = (double)ctas / (double)(waves * slots);
+        if (eff > best + 1e-9) { best = eff; S = cand; }
+        if (eff >= 0.85) { S = cand; break; }
+      }
+    }
+    if (const char* e = getenv("WEDLM_ATTN_SPLITS")) { long long v = atoll(e); if (v > 0) S = v > cap ? cap : v; }
     chunk = (total + S - 1) / S;
     chunk = (chunk + 63) / 64 * 64;
   } else {
@@ -99,7 +114,8 @@ AttnPlan plan_attention(const wedlm_config_t* c) {
     p.part_o_bytes = align_up(rows * c->head_dim * sizeof(float), 256);
     p.part_ml_bytes = align_up(rows * 2 * sizeof(float), 256);
   }
-  p.total_bytes = p.q_rot_bytes + p.part_o_bytes + p.part_ml_bytes;
+  p.order_bytes = align_up((size_t)c->batch * sizeof(int32_t), 256);
+  p.total_bytes = p.q_rot_bytes + p.part_o_bytes + p.part_ml_bytes + p.order_bytes;
   return p;
 }
 
@@ -169,14 +185,15 @@ int wedlm_window_attn(const wedlm_config_t* cfg, const void* q, const void* k, c
   void* q_rot = ws;
   float* part_o = reinterpret_cast<float*>(ws + plan.q_rot_bytes);
   float* part_ml = reinterpret_cast<float*>(ws + plan.q_rot_bytes + plan.part_o_bytes);
+  int32_t* order = reinterpret_cast<int32_t*>(ws + plan.q_rot_bytes + plan.part_o_bytes + plan.part_ml_bytes);
   rc = launch_rope_stage(s, q, k, v, q_rot, k_cache, v_cache, block_table, prefix_len, pos_ids, nullptr, kv_slot_idx,
-                         status, st);
+                         plan.impl == WEDLM_ATTN_TENSOR ? order : nullptr, status, st);
   if (rc != WEDLM_OK) return rc;
   cudaEvent_t ev0 = t_ev_before, ev1 = t_ev_after;
   t_ev_before = t_ev_after = nullptr;
   if (ev0 && cudaEventRecord(ev0, st) != cudaSuccess) return WEDLM_ERR_CUDA;
   if (plan.impl == WEDLM_ATTN_TENSOR)
-    rc = launch_attn_tensor(s, plan, q_rot, k_cache, v_cache, block_table, prefix_len, out, part_o, part_ml, status, st);
+    rc = launch_attn_tensor(s, plan, q_rot, k_cache, v_cache, block_table, prefix_len, order, out, part_o, part_ml, status, st);
   else
     rc = launch_attn_generic(s, plan, q_rot, k_cache, v_cache, block_table, prefix_len, out, part_o, part_ml, status, st);
   if (ev1 && cudaEventRecord(ev1, st) != cudaSuccess) return WEDLM_ERR_CUDA;
@@ -194,7 +211,7 @@ int wedlm_kv_append(const wedlm_config_t* cfg, const void* k, const void* v, con
   if (!k || !v || !k_cache || !v_cache || !block_table || !prefix_len) return WEDLM_ERR_INVALID_ARG;
   if (!aligned16(k) || !aligned16(v) || !aligned16(k_cache) || !aligned16(v_cache)) return WEDLM_ERR_INVALID_ARG;
   return launch_rope_stage(make_shape(cfg), nullptr, k, v, nullptr, k_cache, v_cache, block_table, prefix_len, pos_ids,
-                           count, kv_slot_idx, status, (cudaStream_t)stream);
+                           count, kv_slot_idx, nullptr, status, (cudaStream_t)stream);
 }
 
 size_t wedlm_confidence_workspace_bytes(const wedlm_config_t* cfg) {

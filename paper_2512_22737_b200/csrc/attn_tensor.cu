@@ -53,6 +53,7 @@ struct TensorAttnParams {
   float scale_log2;          // softmax scale * log2(e)
   const int32_t* block_table;
   const int32_t* prefix_len;
+  const int32_t* order;      // sequences by decreasing prefix length, or NULL
   __nv_bfloat16* out;
   float* part_o;
   float* part_ml;
@@ -181,7 +182,8 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   extern __shared__ __align__(1024) uint8_t smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int split = blockIdx.x / p.n_mtiles, mtile = blockIdx.x - split * p.n_mtiles;
-  const int g = blockIdx.y, b = blockIdx.z;
+  const int g = blockIdx.y;
+  const int b = p.order ? p.order[blockIdx.z] : (int)blockIdx.z;     // longest sequences are dispatched first
 
   int P = p.prefix_len[b];
   if (P < 0) { if (p.status && tid == 0) atomicOr(p.status, WEDLM_STATUS_BAD_LENGTH); P = 0; }
@@ -565,8 +567,9 @@ bool attn_tensor_supported(const wedlm_config_t* c) {
 }
 
 int launch_attn_tensor(const Shape& s, const AttnPlan& plan, const void* q_rot, const void* k_cache,
-                       const void* v_cache, const int32_t* block_table, const int32_t* prefix_len, void* out,
-                       float* part_o, float* part_ml, int32_t* status, cudaStream_t st) {
+                       const void* v_cache, const int32_t* block_table, const int32_t* prefix_len,
+                       const int32_t* order, void* out, float* part_o, float* part_ml, int32_t* status,
+                       cudaStream_t st) {
   auto encode = get_encode();
   if (!encode) return WEDLM_ERR_CUDA;
   const int W_t = 128 / s.G;
@@ -599,7 +602,7 @@ int launch_attn_tensor(const Shape& s, const AttnPlan& plan, const void* q_rot, 
   p.B = s.B; p.W = s.W; p.Hq = s.Hq; p.Hkv = s.Hkv; p.G = s.G; p.W_t = W_t; p.n_mtiles = n_mtiles;
   p.n_splits = plan.n_splits; p.chunk = plan.chunk; p.max_pages = s.max_pages; p.num_pages = s.num_pages;
   p.scale_log2 = s.scale * 1.4426950408889634f;
-  p.block_table = block_table; p.prefix_len = prefix_len;
+  p.block_table = block_table; p.prefix_len = prefix_len; p.order = order;
   p.out = (__nv_bfloat16*)out; p.part_o = part_o; p.part_ml = part_ml; p.status = status;
 
   // per device; cheap enough to repeat on every launch

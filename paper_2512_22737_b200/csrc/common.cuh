@@ -52,13 +52,13 @@ int launch_reorder(const Shape& s, const uint8_t* filled, const int32_t* window_
 
 int launch_rope_stage(const Shape& s, const void* q, const void* k, const void* v, void* q_rot, void* k_cache,
                       void* v_cache, const int32_t* block_table, const int32_t* prefix_len, const int32_t* pos_ids,
-                      const int32_t* count, int32_t* kv_slot_idx, int32_t* status, cudaStream_t st);
+                      const int32_t* count, int32_t* kv_slot_idx, int32_t* order, int32_t* status, cudaStream_t st);
 
 struct AttnPlan {
   int impl;            // WEDLM_ATTN_GENERIC or WEDLM_ATTN_TENSOR
   int n_splits;        // key chunks per (sequence, head)
   int chunk;           // keys per chunk (multiple of the page size)
-  size_t q_rot_bytes, part_o_bytes, part_ml_bytes, total_bytes;
+  size_t q_rot_bytes, part_o_bytes, part_ml_bytes, order_bytes, total_bytes;
 };
 AttnPlan plan_attention(const wedlm_config_t* cfg);
 
@@ -68,8 +68,9 @@ int launch_attn_generic(const Shape& s, const AttnPlan& plan, const void* q_rot,
 
 bool attn_tensor_supported(const wedlm_config_t* cfg);
 int launch_attn_tensor(const Shape& s, const AttnPlan& plan, const void* q_rot, const void* k_cache,
-                       const void* v_cache, const int32_t* block_table, const int32_t* prefix_len, void* out,
-                       float* part_o, float* part_ml, int32_t* status, cudaStream_t st);
+                       const void* v_cache, const int32_t* block_table, const int32_t* prefix_len,
+                       const int32_t* order, void* out, float* part_o, float* part_ml, int32_t* status,
+                       cudaStream_t st);
 
 int launch_attn_merge(const Shape& s, const AttnPlan& plan, const int32_t* prefix_len, const float* part_o,
                       const float* part_ml, void* out, cudaStream_t st);

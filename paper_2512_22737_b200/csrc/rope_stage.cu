@@ -18,7 +18,7 @@ rope_stage_kernel(Shape s, const InvFreq inv_freq, const T* __restrict__ q, cons
                   T* __restrict__ q_rot, T* __restrict__ k_cache, T* __restrict__ v_cache,
                   const int32_t* __restrict__ block_table, const int32_t* __restrict__ prefix_len,
                   const int32_t* __restrict__ pos_ids, const int32_t* __restrict__ count,
-                  int32_t* __restrict__ kv_slot_idx, int32_t* status) {
+                  int32_t* __restrict__ kv_slot_idx, int32_t* __restrict__ order, int32_t* status) {
   extern __shared__ float cs_sn[];  // [D/2] cos, [D/2] sin
   const int i = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
   const int D = s.D, half = D / 2;
@@ -41,6 +41,23 @@ rope_stage_kernel(Shape s, const InvFreq inv_freq, const T* __restrict__ q, cons
     for (int d = tid; d < half; d += blockDim.x) { cs[d] = 1.f; sn[d] = 0.f; }
   }
   __syncthreads();
+
+  // Side job of the blocks of row 0: rank the sequences by prefix length (longest first, ties by
+  // index) so that the attention kernel can start the longest work first.  order[rank] = b.
+  if (order != nullptr && i == 0) {
+    __shared__ int rank_acc;
+    if (tid == 0) rank_acc = 0;
+    __syncthreads();
+    const int mine = prefix_len[b];
+    int cnt = 0;
+    for (int o = tid; o < s.B; o += blockDim.x) {
+      const int other = prefix_len[o];
+      cnt += (other > mine || (other == mine && o < b)) ? 1 : 0;
+    }
+    if (cnt) atomicAdd(&rank_acc, cnt);
+    __syncthreads();
+    if (tid == 0) order[rank_acc] = b;
+  }
 
   const size_t row = (size_t)b * s.W + i;
   if (q != nullptr) {
@@ -80,7 +97,7 @@ rope_stage_kernel(Shape s, const InvFreq inv_freq, const T* __restrict__ q, cons
 
 int launch_rope_stage(const Shape& s, const void* q, const void* k, const void* v, void* q_rot, void* k_cache,
                       void* v_cache, const int32_t* block_table, const int32_t* prefix_len, const int32_t* pos_ids,
-                      const int32_t* count, int32_t* kv_slot_idx, int32_t* status, cudaStream_t st) {
+                      const int32_t* count, int32_t* kv_slot_idx, int32_t* order, int32_t* status, cudaStream_t st) {
   dim3 grid(s.W, s.B);
   size_t smem = (size_t)s.D * sizeof(float);
   InvFreq inv_freq;
@@ -90,12 +107,12 @@ int launch_rope_stage(const Shape& s, const void* q, const void* k, const void* 
     using T = __nv_bfloat16;
     rope_stage_kernel<T><<<grid, 128, smem, st>>>(s, inv_freq, (const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_cache,
                                                   (T*)v_cache, block_table, prefix_len, pos_ids, count, kv_slot_idx,
-                                                  status);
+                                                  order, status);
   } else {
     using T = float;
     rope_stage_kernel<T><<<grid, 128, smem, st>>>(s, inv_freq, (const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_cache,
                                                   (T*)v_cache, block_table, prefix_len, pos_ids, count, kv_slot_idx,
-                                                  status);
+                                                  order, status);
   }
   count_launch();
   return cuda_ok(cudaGetLastError());
