@@ -29,9 +29,11 @@ METRIC = "committed_tokens_per_s"
 UNIT = "tokens/s"
 L2_BYTES = 126 * 1024 * 1024
 
-# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from
-# one ncu capture; the summaries under profiles/ give the commands).  None = not captured.
-NCU_TRAFFIC_BYTES = {}
+# DRAM traffic of the dominant kernel as a multiple of its algorithmic bytes
+# (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture on a batch-16 case of the same
+# shapes; profiles/attn_tensor_kernel_cfg3_batch16.md gives the command).  Traffic grows with the
+# tokens streamed, so the ratio is applied to the launch that is timed.  Missing = not captured.
+NCU_TRAFFIC_RATIO = {"cfg3_batched:auto": 1.011, "cfg3_batched:tensor": 1.011}
 
 
 def log(*a):
@@ -437,7 +439,9 @@ def run_product(args):
             "roofline": {"bound": "hbm", "kernel": "window attention", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                          "frac_of_nominal_8TBps": achieved / 8000.0,
-                         "traffic": NCU_TRAFFIC_BYTES.get(key), "kernel_ms": attn_ms,
+                         "traffic": (NCU_TRAFFIC_RATIO[key] * bts["attn_kernel"] if key in NCU_TRAFFIC_RATIO and not args.batch else None),
+                         "traffic_note": "ncu dram bytes of a batch-16 capture scaled by algorithmic bytes",
+                         "kernel_ms": attn_ms,
                          "algorithmic_bytes": bts["attn_kernel"]},
             "cpu_baseline": cpu,
             "other_workloads": others,
