@@ -329,6 +329,26 @@ def time_e2e(wl, steps, warmup, sampler=None):
     return ms, committed, h2d, d2h
 
 
+def rank_seed(rank: int) -> int:
+    """Every rank draws its own batch of the same shape (weak scaling over independent sequences)."""
+    from workloads import BASE_SEED
+    return BASE_SEED + rank
+
+
+def reduce_over_ranks(times_ms, counts, device):
+    """Job-level figures from per-rank ones: MAX over ranks of every time, SUM over ranks of every
+    count.  Works on any backend (NCCL on the GPUs, gloo in the CPU tests); a single process returns
+    its own values."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    c = torch.tensor(list(counts), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t.tolist()], [float(x) for x in c.tolist()]
+
+
 def run_product(args):
     import torch
     import torch.distributed as dist
@@ -352,7 +372,7 @@ def run_product(args):
 
     sampler = ClockSampler(local) if rank == 0 else None
     n_state = args.steps + args.warmup
-    wl = Workload(args.workload, BASE_SEED + rank, args.attn, n_state, args.batch)
+    wl = Workload(args.workload, rank_seed(rank), args.attn, n_state, args.batch)
     if sampler:
         sampler.start()
 
@@ -364,28 +384,14 @@ def run_product(args):
     barrier()
     ms, attn_ms, committed, launches = time_workload(wl, args.steps, args.warmup, sampler)
     barrier()
-    t = torch.tensor([ms, attn_ms, float(committed)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        tmax = t.clone()
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        tsum = t.clone()
-        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
-        ms, attn_ms, committed_total = float(tmax[0]), float(tmax[1]), float(tsum[2])
-    else:
-        committed_total = float(committed)
+    (ms, attn_ms), (committed_total,) = reduce_over_ranks([ms, attn_ms], [committed], "cuda")
     assert int(wl.step.status.item()) == 0, "device status word set during the benchmark"
 
     if args.no_e2e:
         e2e_ms, e2e_committed, h2d, d2h = float("nan"), 0, 0, 0
     else:
         e2e_ms, e2e_committed, h2d, d2h = time_e2e(wl, max(3, min(args.steps, 10)), 3, sampler)
-    te = torch.tensor([e2e_ms, float(e2e_committed)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        tm = te.clone()
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        tsu = te.clone()
-        dist.all_reduce(tsu, op=dist.ReduceOp.SUM)
-        e2e_ms, e2e_committed = float(tm[0]), float(tsu[1])
+    (e2e_ms,), (e2e_committed,) = reduce_over_ranks([e2e_ms], [e2e_committed], "cuda")
 
     others = {}
     cpu = None

@@ -1,0 +1,164 @@
+"""Streaming Parallel Decoding (Algorithm 1) as a loop around the library's step calls.
+
+Harness for the end-to-end configuration: a random-init pre-norm decoder (RMSNorm, GQA attention,
+SwiGLU) whose dense projections are plain library GEMMs (torch.matmul), while every step of the
+decoding hot path runs in this package's kernels: wedlm_reorder, wedlm_window_attn (RoPE at the
+logical ids, staging into the paged cache, causal window attention), wedlm_confidence_commit
+(confidence, Eq. 11 selection, commit / refill) and wedlm_window_refill (prefill commit).
+
+Window state, block tables and caches stay on the device for the whole generation; the host reads
+back only the committed tokens of each step.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as w
+
+
+def _dev(x: np.ndarray) -> torch.Tensor:
+    return w.to_device(x)
+
+
+class StreamingDecoder:
+    def __init__(self, mcfg, weights: Dict[str, np.ndarray], *, batch: int, window: int, max_total_len: int,
+                 conf_mode: str = "entropy", tau: float = 0.3, lam: float = 0.1, maxprob_thr: float = 0.9,
+                 tilt: float = 0.0, target: Optional[np.ndarray] = None, page_size: int = 16,
+                 attn_impl: str = "auto", seed: int = 0):
+        self.m = mcfg
+        self.B, self.W = batch, window
+        self.dtype = torch.bfloat16 if mcfg.dtype == "bf16" else torch.float32
+        self.wt = {k: _dev(v) for k, v in weights.items()}
+        self.tilt = tilt
+        self.target = None if target is None else torch.from_numpy(target.astype(np.int64)).cuda()
+        # paged caches, one pair per layer, sharing one block table (scattered pages)
+        pages_per_seq = (max_total_len + window + page_size - 1) // page_size
+        self.num_pages = batch * pages_per_seq + 3
+        g = np.random.default_rng(seed)
+        order = g.permutation(self.num_pages).astype(np.int32)
+        self.block_table = torch.from_numpy(order[: batch * pages_per_seq].reshape(batch, pages_per_seq).copy()).cuda()
+        shape = (self.num_pages, mcfg.n_kv_heads, page_size, mcfg.head_dim)
+        self.k_cache = [torch.zeros(shape, dtype=self.dtype, device="cuda") for _ in range(mcfg.n_layers)]
+        self.v_cache = [torch.zeros(shape, dtype=self.dtype, device="cuda") for _ in range(mcfg.n_layers)]
+        self.cfg = w.make_config(
+            batch=batch, window=window, n_q_heads=mcfg.n_q_heads, n_kv_heads=mcfg.n_kv_heads, head_dim=mcfg.head_dim,
+            page_size=page_size, max_pages_per_seq=pages_per_seq, num_pages=self.num_pages, vocab=mcfg.vocab,
+            dtype=mcfg.dtype, rope_theta=mcfg.rope_theta, conf_mode=conf_mode, tau=tau, lam=lam,
+            maxprob_thr=maxprob_thr, mask_token_id=mcfg.mask_token_id, max_prefix_len=max_total_len,
+            attn_impl=attn_impl)
+        self.step_bufs = w.DecodeStep(self.cfg)
+        i32 = dict(dtype=torch.int32, device="cuda")
+        self.window_tokens = torch.full((batch, window), mcfg.mask_token_id, **i32)
+        self.filled = torch.zeros(batch, window, dtype=torch.uint8, device="cuda")
+        self.prefix_len = torch.zeros(batch, **i32)
+        self.window_len = torch.zeros(batch, **i32)
+        self.budget = torch.zeros(batch, **i32)
+        self.n_fwd = 0
+        self.steps = 0
+
+    # ------------------------------------------------------------------ dense parts (library GEMMs)
+    def _rms(self, x: torch.Tensor, gain: torch.Tensor) -> torch.Tensor:
+        xf = x.float()
+        y = xf * torch.rsqrt(xf.pow(2).mean(-1, keepdim=True) + self.m.rms_eps)
+        return (y * gain.float()).to(self.dtype)
+
+    def forward(self, capture_layer: Optional[int] = None):
+        """Causal forward of the reordered window on top of the cache -> logits [B, W, V]."""
+        s, m = self.step_bufs, self.m
+        B, W = self.B, self.W
+        s.reorder(self.filled, self.window_tokens, self.prefix_len, self.window_len)
+        h = self.wt["embed"][s.tokens_phys.long()]                       # [B, W, H]
+        cap = None
+        for l in range(m.n_layers):
+            a = self._rms(h, self.wt[f"l{l}.norm1"])
+            q = (a @ self.wt[f"l{l}.wq"]).view(B, W, m.n_q_heads, m.head_dim).contiguous()
+            k = (a @ self.wt[f"l{l}.wk"]).view(B, W, m.n_kv_heads, m.head_dim).contiguous()
+            v = (a @ self.wt[f"l{l}.wv"]).view(B, W, m.n_kv_heads, m.head_dim).contiguous()
+            if capture_layer == l:
+                cap = dict(q=q.clone(), k=k.clone(), v=v.clone(), k_cache=self.k_cache[l].clone(),
+                           v_cache=self.v_cache[l].clone())
+            s.attention(q, k, v, self.k_cache[l], self.v_cache[l], self.block_table, self.prefix_len)
+            if capture_layer == l:
+                cap["out"] = s.out.clone()
+                cap["kv_slot_idx"] = s.kv_slot_idx.clone()
+            h = h + s.out.view(B, W, -1) @ self.wt[f"l{l}.wo"]
+            mm = self._rms(h, self.wt[f"l{l}.norm2"])
+            h = h + (torch.nn.functional.silu(mm @ self.wt[f"l{l}.wg"]) * (mm @ self.wt[f"l{l}.wu"])) @ self.wt[f"l{l}.wd"]
+        logits = self._rms(h, self.wt["norm_f"]) @ self.wt["lm_head"]
+        if self.tilt != 0.0 and self.target is not None:
+            pos = s.pos_ids.long().clamp_(max=self.target.shape[1] - 1)
+            idx = self.target.gather(1, pos)                                 # [B, W] target id at each row's position
+            logits.scatter_add_(2, idx.unsqueeze(-1), torch.full((B, W, 1), self.tilt, dtype=self.dtype, device="cuda"))
+        return logits.contiguous(), cap
+
+    # ------------------------------------------------------------------ Algorithm 1
+    def prefill(self, prompt: np.ndarray) -> None:
+        """Push the prompt through the layers W tokens at a time (windows of filled slots); each
+        window is committed whole, which is just prefix_len += n."""
+        B, W = self.B, self.W
+        P = prompt.shape[1]
+        prompt_dev = torch.from_numpy(prompt.astype(np.int32)).cuda()
+        zero_budget = torch.zeros(B, dtype=torch.int32, device="cuda")
+        for at in range(0, P, W):
+            n = min(W, P - at)
+            self.window_tokens.fill_(self.m.mask_token_id)
+            self.window_tokens[:, :n] = prompt_dev[:, at:at + n]
+            self.filled.zero_()
+            self.filled[:, :n] = 1
+            self.window_len.fill_(n)
+            self.forward()
+            zero_budget.zero_()
+            w.wedlm_window_refill(self.cfg, self.step_bufs.n_commit, self.window_tokens, self.filled, self.prefix_len,
+                                  self.window_len, zero_budget, None, None)
+
+    def start(self, max_new_tokens: int) -> None:
+        n0 = min(self.W, max_new_tokens)
+        self.window_tokens.fill_(self.m.mask_token_id)
+        self.filled.zero_()
+        self.window_len.fill_(n0)
+        self.budget.fill_(max_new_tokens - n0)
+        self.n_fwd = 0
+        self.steps = 0
+
+    def step(self, capture_layer: Optional[int] = None):
+        """One iteration of Algorithm 1.  Returns (committed_count, committed_tokens) device tensors
+        (and the captured tensors of one layer when asked)."""
+        s = self.step_bufs
+        active = int(self.window_len.sum().item()) if capture_layer is not None else None
+        snap = None
+        if capture_layer is not None:
+            snap = dict(filled=self.filled.clone(), window_tokens=self.window_tokens.clone(),
+                        prefix_len=self.prefix_len.clone(), window_len=self.window_len.clone(),
+                        budget=self.budget.clone())
+        logits, cap = self.forward(capture_layer)
+        s.confidence_commit(logits, self.window_tokens, self.filled, self.prefix_len, self.window_len, self.budget)
+        self.steps += 1
+        if capture_layer is not None:
+            cap.update(snap)
+            cap["logits"] = logits
+            cap["active"] = active
+            return s.committed_count, s.committed_tokens, cap
+        return s.committed_count, s.committed_tokens
+
+    def generate(self, max_new_tokens: int, max_steps: int = 1_000_000) -> Dict[str, object]:
+        """Runs until every window is empty.  Returns the committed text per sequence, the number of
+        steps and the prefix cacheability p_cache = N_gen / N_fwd (Eq. 4)."""
+        self.start(max_new_tokens)
+        ys: List[List[int]] = [[] for _ in range(self.B)]
+        commits_per_step = []
+        while self.steps < max_steps:
+            wl = self.window_len.cpu()
+            if int(wl.sum()) == 0:
+                break
+            self.n_fwd += int(wl.sum())
+            cc, ct = self.step()
+            cc_h, ct_h = cc.cpu().numpy(), ct.cpu().numpy()
+            for b in range(self.B):
+                ys[b].extend(ct_h[b, : cc_h[b]].tolist())
+            commits_per_step.append(int(cc_h.sum()))
+        n_gen = sum(len(y) for y in ys)
+        return dict(y=ys, steps=self.steps, n_fwd=self.n_fwd, p_cache=(n_gen / self.n_fwd if self.n_fwd else 0.0),
+                    commits_per_step=commits_per_step)
