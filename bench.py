@@ -459,6 +459,76 @@ def run_product(args):
     return 0
 
 
+# ----------------------------------------------------------------------------------------------
+# end-to-end streaming decode loop (the 4-layer configuration); not the default bench line
+# ----------------------------------------------------------------------------------------------
+def run_loop(args):
+    """Random-init 4-layer model of Qwen3-8B width, batch 16, 512-token prompt, 1024 new tokens per
+    sequence, LM-head logits tilted toward a seeded target sequence.  Generated tokens/s, steps and
+    p_cache (Eq. 4) for W = 16 against the same harness at W = 1 and W = 2, for every tilt."""
+    import torch
+    from paper_2512_22737_b200 import build as b
+    from paper_2512_22737_b200.loop import StreamingDecoder
+    from workloads.model import QWEN_4L, make_prompts_and_targets
+    b.build()
+    torch.cuda.set_device(0)
+    m = QWEN_4L
+    B, P, N = args.loop_batch, 512, args.loop_new_tokens
+    g = torch.Generator(device="cuda").manual_seed(251222737)
+    H, F = m.hidden, m.ffn
+
+    def mat(*shape):
+        return (torch.randn(*shape, generator=g, device="cuda", dtype=torch.float32) * m.init_std).to(torch.bfloat16)
+
+    class DeviceWeights(dict):
+        pass
+    wts = DeviceWeights(embed=mat(m.vocab, H), lm_head=mat(H, m.vocab), norm_f=torch.ones(H, device="cuda", dtype=torch.bfloat16))
+    for l in range(m.n_layers):
+        wts[f"l{l}.norm1"] = torch.ones(H, device="cuda", dtype=torch.bfloat16)
+        wts[f"l{l}.norm2"] = torch.ones(H, device="cuda", dtype=torch.bfloat16)
+        wts[f"l{l}.wq"] = mat(H, m.n_q_heads * m.head_dim)
+        wts[f"l{l}.wk"] = mat(H, m.n_kv_heads * m.head_dim)
+        wts[f"l{l}.wv"] = mat(H, m.n_kv_heads * m.head_dim)
+        wts[f"l{l}.wo"] = mat(m.n_q_heads * m.head_dim, H)
+        wts[f"l{l}.wg"] = mat(H, F)
+        wts[f"l{l}.wu"] = mat(H, F)
+        wts[f"l{l}.wd"] = mat(F, H)
+    pt = make_prompts_and_targets(m, B, P, N)
+    results = []
+    lse0 = None
+    for W in args.loop_windows:
+        for tilt_name, tilt in args.loop_tilts:
+            dec = StreamingDecoder(m, {}, batch=B, window=W, max_total_len=P + N, tau=0.3, lam=0.1, tilt=0.0,
+                                   target=pt["target"])
+            dec.wt = wts
+            dec.prefill(pt["prompt"])
+            if lse0 is None:                    # log-sum-exp of the untilted logits, measured once
+                dec.start(N)
+                lg, _ = dec.forward()
+                lse0 = float(torch.logsumexp(lg[:, 0].float(), dim=-1).mean().item())
+            dec.tilt = tilt if tilt_name == "literal" else lse0 + tilt
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            out = dec.generate(N)
+            torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+            n_gen = sum(len(y) for y in out["y"])
+            on_target = sum(int(out["y"][bb] == pt["target"][bb, P:P + N].tolist()) for bb in range(B))
+            results.append({"window": W, "tilt": f"{tilt_name}+{tilt:g}", "tokens_per_s": n_gen / dt, "seconds": dt,
+                            "steps": out["steps"], "tokens_per_step_per_seq": n_gen / B / max(out["steps"], 1),
+                            "p_cache": out["p_cache"], "sequences_equal_to_target": on_target})
+            log(results[-1])
+            del dec
+            torch.cuda.empty_cache()
+    line = {"metric": "generated_tokens_per_s", "unit": "tokens/s", "n_gpus": 1, "data": "synthetic", "dtype": "bf16",
+            "config": {"workload": "cfg5_loop", "batch": B, "prompt": P, "new_tokens": N, "layers": m.n_layers,
+                       "hidden": H, "lse_of_untilted_logits": lse0,
+                       "timing": "host wall clock around generate(), includes the per-step read-back of commits"},
+            "results": results}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -471,7 +541,14 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing (profiling runs)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling runs)")
+    ap.add_argument("--loop-batch", type=int, default=16)
+    ap.add_argument("--loop-new-tokens", type=int, default=1024)
+    ap.add_argument("--loop-windows", type=lambda s: [int(x) for x in s.split(",")], default=[16, 2, 1])
+    ap.add_argument("--loop-tilts", type=lambda s: [(t.split(":")[0], float(t.split(":")[1])) for t in s.split(",")],
+                    default=[("literal", 2.0), ("literal", 4.0), ("literal", 8.0), ("lse", 2.0), ("lse", 4.0), ("lse", 8.0)])
     args = ap.parse_args()
+    if args.workload == "cfg5_loop":
+        return run_loop(args)
     args.warmup = max(args.warmup, 3) if args.impl == "product" else args.warmup
     if args.impl == "reference":
         return run_reference(args)

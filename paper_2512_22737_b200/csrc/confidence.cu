@@ -400,8 +400,9 @@ struct ConfParams {
   float tau, lambda, thr;
 };
 
-// One warp per sequence.
-__global__ void __launch_bounds__(32)
+// One block per sequence with up to one warp per window row.  Each warp merges the chunk partials of
+// whole rows (lanes over chunks, double precision), then warp 0 runs the selection and the window update.
+__global__ void __launch_bounds__(1024)
 conf_commit_kernel(ConfParams p, const float4* __restrict__ part, const int32_t* __restrict__ perm,
                    const int32_t* __restrict__ n_filled, const int32_t* __restrict__ n_commit,
                    int32_t* window_tokens, uint8_t* filled, int32_t* prefix_len, int32_t* window_len,
@@ -415,19 +416,19 @@ conf_commit_kernel(ConfParams p, const float4* __restrict__ part, const int32_t*
   uint8_t* fil_s = reinterpret_cast<uint8_t*>(tok_s + W);     // [W] logical
   uint8_t* pass = fil_s + W;                                  // [W] per mask k
 
-  const int b = blockIdx.x, lane = threadIdx.x;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const size_t o = (size_t)b * W;
   const int L = window_len ? min(max(window_len[b], 0), W) : W;
   const int nf = min(max(n_filled[b], 0), L);
   const int n_mask = L - nf;
   const float qnan = __int_as_float(0x7fc00000);
 
-  for (int j = lane; j < W; j += 32) {
+  for (int j = tid; j < W; j += blockDim.x) {
     tok_s[j] = window_tokens[o + j];
     fil_s[j] = (j < L && filled[o + j]) ? 1 : 0;
   }
   // rows that are not active masks carry no statistics
-  for (int i = lane; i < W; i += 32) {
+  for (int i = tid; i < W; i += blockDim.x) {
     if (i < nf || i >= L) {
       if (argmax) argmax[o + i] = -1;
       if (maxprob) maxprob[o + i] = qnan;
@@ -436,51 +437,70 @@ conf_commit_kernel(ConfParams p, const float4* __restrict__ part, const int32_t*
     }
   }
   const int j0 = n_mask > 0 ? perm[o + nf] : 0;
-  int n_pass = 0;
-  for (int k = lane; k < n_mask; k += 32) {
+  for (int k = warp; k < n_mask; k += (int)(blockDim.x >> 5)) {
     const int i = nf + k;
     const float4* pr = part + (o + i) * p.n_chunks;
+    // arg-max over the chunks: larger maximum wins, equal maxima keep the lower token index
     float m = -CUDART_INF_F;
     int a = 0x7fffffff;
-    for (int c = 0; c < p.n_chunks; ++c) {
-      float4 v = pr[c];
-      argmax_combine(m, a, v.x, __float_as_int(v.w));     // chunks ascend in index, ties keep the lower
+    float4 v0 = make_float4(-CUDART_INF_F, 0.f, 0.f, __int_as_float(0x7fffffff));   // this lane's first chunk
+    if (lane < p.n_chunks) v0 = pr[lane];
+    argmax_combine(m, a, v0.x, __float_as_int(v0.w));
+    for (int c = lane + 32; c < p.n_chunks; c += 32) {
+      const float4 v = pr[c];
+      argmax_combine(m, a, v.x, __float_as_int(v.w));
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float om = __shfl_xor_sync(0xffffffffu, m, off);
+      const int oa = __shfl_xor_sync(0xffffffffu, a, off);
+      argmax_combine(m, a, om, oa);
     }
     double s = 0.0, t = 0.0;
-    for (int c = 0; c < p.n_chunks; ++c) {
-      float4 v = pr[c];
+    for (int c = lane; c < p.n_chunks; c += 32) {
+      const float4 v = (c == lane) ? v0 : pr[c];
       if (v.x > -CUDART_INF_F) {
-        double dm = (double)v.x - (double)m;
-        double w = exp(dm);
-        s += w * (double)v.y;
-        t += w * ((double)v.z + dm * (double)v.y);
+        const double dm = (double)v.x - (double)m;
+        const double wgt = exp(dm);
+        s += wgt * (double)v.y;
+        t += wgt * ((double)v.z + dm * (double)v.y);
       }
     }
-    const double ln_s = log(s);
-    const double H = ln_s - t / s;
-    const double pmax = 1.0 / s;
-    if (argmax) argmax[o + i] = a;
-    if (maxprob) maxprob[o + i] = (float)pmax;
-    if (entropy) entropy[o + i] = (float)H;
-    if (lse) lse[o + i] = (float)((double)m + ln_s);
-    const int j = perm[o + i];
-    double sc;
-    bool ok;
-    if (p.conf_mode == WEDLM_CONF_ENTROPY) {
-      sc = H + (double)p.lambda * (double)(j - j0);           // Eq. 11
-      ok = sc <= (double)p.tau;
-    } else {
-      sc = -pmax;
-      ok = pmax >= (double)p.thr;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      s += __shfl_xor_sync(0xffffffffu, s, off);
+      t += __shfl_xor_sync(0xffffffffu, t, off);
     }
-    score[k] = sc;
-    am[k] = a;
-    pass[k] = ok ? 1 : 0;
-    n_pass += ok ? 1 : 0;
+    if (lane == 0) {
+      const double ln_s = log(s);
+      const double H = ln_s - t / s;
+      const double pmax = 1.0 / s;
+      if (argmax) argmax[o + i] = a;
+      if (maxprob) maxprob[o + i] = (float)pmax;
+      if (entropy) entropy[o + i] = (float)H;
+      if (lse) lse[o + i] = (float)((double)m + ln_s);
+      const int j = perm[o + i];
+      double sc;
+      bool ok;
+      if (p.conf_mode == WEDLM_CONF_ENTROPY) {
+        sc = H + (double)p.lambda * (double)(j - j0);           // Eq. 11
+        ok = sc <= (double)p.tau;
+      } else {
+        sc = -pmax;
+        ok = pmax >= (double)p.thr;
+      }
+      score[k] = sc;
+      am[k] = a;
+      pass[k] = ok ? 1 : 0;
+    }
   }
+  __syncthreads();
+  if (warp != 0) return;
+
+  int n_pass = 0;
+  for (int k = lane; k < n_mask; k += 32) n_pass += pass[k];
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) n_pass += __shfl_xor_sync(0xffffffffu, n_pass, off);
-  __syncwarp();
   if (n_pass == 0 && n_mask > 0) {
     // nothing passed: fill the single best-scoring mask, leftmost on ties
     double best = CUDART_INF;
@@ -574,7 +594,9 @@ int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* log
   if (cudaGetLastError() != cudaSuccess) return WEDLM_ERR_CUDA;
   ConfParams p{s.W, n_chunks, cfg->conf_mode, cfg->mask_token_id, cfg->tau, cfg->lambda, cfg->maxprob_thr};
   size_t smem = (size_t)s.W * (sizeof(double) + 2 * sizeof(int) + 2);
-  conf_commit_kernel<<<s.B, 32, smem, st>>>(p, part, perm, n_filled, n_commit, window_tokens, filled, prefix_len,
+  int commit_threads = 32 * s.W;
+  commit_threads = commit_threads < 128 ? 128 : (commit_threads > 1024 ? 1024 : commit_threads);
+  conf_commit_kernel<<<s.B, commit_threads, smem, st>>>(p, part, perm, n_filled, n_commit, window_tokens, filled, prefix_len,
                                             window_len, remaining_budget, argmax, maxprob, entropy, lse,
                                             committed_tokens, committed_count, filled_count);
   count_launch();

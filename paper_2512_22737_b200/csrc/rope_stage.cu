@@ -10,6 +10,25 @@ namespace wedlm {
 // theta^(-2d/D) for d < D/2, computed on the host in double and passed by value (D <= 256).
 struct InvFreq { double v[128]; };
 
+// Rotate eight bf16 pairs (a_e, c_e) held in two 16-byte vectors: a' = a cos - c sin, c' = c cos + a sin.
+__device__ __forceinline__ void rotate8(const uint4& a, const uint4& c, const float* cs, const float* sn, uint4& oa,
+                                        uint4& oc) {
+  const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
+  uint32_t ra[4], rc[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float a0 = __uint_as_float(aw[e] << 16), a1 = __uint_as_float(aw[e] & 0xffff0000u);
+    const float c0 = __uint_as_float(cw[e] << 16), c1 = __uint_as_float(cw[e] & 0xffff0000u);
+    const float cs0 = cs[2 * e], cs1 = cs[2 * e + 1], sn0 = sn[2 * e], sn1 = sn[2 * e + 1];
+    __nv_bfloat162 va = __floats2bfloat162_rn(a0 * cs0 - c0 * sn0, a1 * cs1 - c1 * sn1);
+    __nv_bfloat162 vc = __floats2bfloat162_rn(c0 * cs0 + a0 * sn0, c1 * cs1 + a1 * sn1);
+    ra[e] = *reinterpret_cast<uint32_t*>(&va);
+    rc[e] = *reinterpret_cast<uint32_t*>(&vc);
+  }
+  oa = make_uint4(ra[0], ra[1], ra[2], ra[3]);
+  oc = make_uint4(rc[0], rc[1], rc[2], rc[3]);
+}
+
 // grid (W, B); one block per (physical row i, sequence b).  Angles are formed in double so that
 // positions of tens of thousands keep full fp32 accuracy after the range reduction.
 template <typename T>
@@ -60,6 +79,41 @@ rope_stage_kernel(Shape s, const InvFreq inv_freq, const T* __restrict__ q, cons
   }
 
   const size_t row = (size_t)b * s.W + i;
+  if (sizeof(T) == 2 && s.rope_style == 0 && (D % 16) == 0) {
+    // bf16, rotate-half pairing: 16-byte loads of the two halves of each head, 16-byte stores
+    const int vph = half / 8;                                   // vectors per half head
+    if (q != nullptr) {
+      const uint4* src = reinterpret_cast<const uint4*>(q + row * s.Hq * D);
+      uint4* dst = reinterpret_cast<uint4*>(q_rot + row * s.Hq * D);
+      for (int idx = tid; idx < s.Hq * vph; idx += blockDim.x) {
+        const int h = idx / vph, j = idx - h * vph;
+        uint4 oa, oc;
+        rotate8(src[h * 2 * vph + j], src[h * 2 * vph + vph + j], cs + 8 * j, sn + 8 * j, oa, oc);
+        dst[h * 2 * vph + j] = oa;
+        dst[h * 2 * vph + vph + j] = oc;
+      }
+    }
+    const int n_rows = count ? count[b] : s.W;
+    long long slot = -1;
+    if (i < n_rows) slot = cache_slot(block_table, b, prefix_len[b] + i, s.page, s.max_pages, s.num_pages, status);
+    if (kv_slot_idx && tid == 0) kv_slot_idx[row] = (int32_t)slot;
+    if (slot < 0) return;
+    const uint4* ksrc = reinterpret_cast<const uint4*>(k + row * s.Hkv * D);
+    const uint4* vsrc = reinterpret_cast<const uint4*>(v + row * s.Hkv * D);
+    for (int idx = tid; idx < s.Hkv * vph; idx += blockDim.x) {
+      const int g = idx / vph, j = idx - g * vph;
+      uint4 oa, oc;
+      rotate8(ksrc[g * 2 * vph + j], ksrc[g * 2 * vph + vph + j], cs + 8 * j, sn + 8 * j, oa, oc);
+      uint4* kd = reinterpret_cast<uint4*>(k_cache + cache_offset(slot, g, s.page, s.Hkv, D));
+      kd[j] = oa;
+      kd[vph + j] = oc;
+    }
+    for (int idx = tid; idx < s.Hkv * 2 * vph; idx += blockDim.x) {
+      const int g = idx / (2 * vph), j = idx - g * 2 * vph;
+      reinterpret_cast<uint4*>(v_cache + cache_offset(slot, g, s.page, s.Hkv, D))[j] = vsrc[idx];
+    }
+    return;
+  }
   if (q != nullptr) {
     const T* src = q + row * s.Hq * D;
     T* dst = q_rot + row * s.Hq * D;
