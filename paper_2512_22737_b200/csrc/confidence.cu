@@ -35,13 +35,12 @@ __device__ __forceinline__ void unpack16(const uint4& u, float (&x)[4]) {
 }
 
 // Packed fp32x2 arithmetic of sm_100 (two lanes per instruction).
-__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
-  unsigned long long r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {     // a register pair, no instruction
+  return ((unsigned long long)__float_as_uint(hi) << 32) | (unsigned long long)__float_as_uint(lo);
 }
 __device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+  lo = __uint_as_float((unsigned)(v & 0xffffffffull));
+  hi = __uint_as_float((unsigned)(v >> 32));
 }
 __device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
   unsigned long long d;
@@ -186,8 +185,13 @@ conf_partial_kernel(int W, int V, int n_chunks, const T* __restrict__ logits, co
 // asynchronous copies (one 16 KB copy per item, completion on an mbarrier), so that the bytes in
 // flight per SM do not depend on registers.  Same chunking and partial layout as conf_partial_kernel.
 // ------------------------------------------------------------------------------------------------
-constexpr int kStreamStages = 4;
-constexpr int kStreamChunk = kConfThreads * kConfVecs * 8;          // 8192 bf16 = 16 KB
+constexpr int kStreamStages = 2;                                    // power of two (stage = n & (stages - 1))
+constexpr int kStreamBlocksPerSM = 6;                               // 32 KB ring each
+constexpr int kStreamThreads = 128;                                 // consumer threads per block
+constexpr int kStreamVecs = 8;                                      // 16-byte vectors per thread and item
+constexpr int kStreamChunk = kStreamThreads * kStreamVecs * 8;      // 8192 bf16 = 16 KB, same chunking as pass 1 above
+static_assert((kStreamStages & (kStreamStages - 1)) == 0, "stage index uses a mask");
+static_assert(kStreamChunk == kConfThreads * kConfVecs * 8, "both pass-1 kernels must cut rows the same way");
 constexpr uint32_t kStreamSpin = 1u << 22;
 
 __device__ __forceinline__ uint32_t cs_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -204,12 +208,12 @@ __device__ __forceinline__ bool cs_mbar_wait(uint32_t bar, uint32_t parity) {
   return false;
 }
 
-__device__ __forceinline__ void cs_consumer_sync() {     // the 256 consumer threads only
-  asm volatile("bar.sync 1, 256;" ::: "memory");
+__device__ __forceinline__ void cs_consumer_sync() {     // the consumer threads only
+  asm volatile("bar.sync 1, %0;" ::"n"(kStreamThreads) : "memory");
 }
 
-// block = 8 consumer warps (threads 0..255) + 1 producer warp (lane 0 of warp 8 issues the copies)
-__global__ void __launch_bounds__(kConfThreads + 32)
+// block = 4 consumer warps + 1 producer warp (its lane 0 issues the copies)
+__global__ void __launch_bounds__(kStreamThreads + 32)
 conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv_bfloat16* __restrict__ logits,
                    const int32_t* __restrict__ n_filled, const int32_t* __restrict__ window_len,
                    float4* __restrict__ part) {
@@ -217,10 +221,10 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
   unsigned char* stage_mem = cs_smem;                                       // kStreamStages x 16 KB
   uint64_t* full = reinterpret_cast<uint64_t*>(cs_smem + kStreamStages * kStreamChunk * 2);
   uint64_t* empty = full + kStreamStages;
-  volatile long long* item_of = reinterpret_cast<volatile long long*>(empty + kStreamStages);
-  __shared__ float fm[kConfThreads / 32];
-  __shared__ float fs[kConfThreads / 32];
-  __shared__ float ft[kConfThreads / 32];
+  volatile int2* item_of = reinterpret_cast<volatile int2*>(empty + kStreamStages);   // (row, chunk) or (-1, -1)
+  __shared__ float fm[kStreamThreads / 32];
+  __shared__ float fs[kStreamThreads / 32];
+  __shared__ float ft[kStreamThreads / 32];
   __shared__ int fa;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   long long cursor = blockIdx.x;                     // next candidate item of this block (producer only)
@@ -233,7 +237,7 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
       const long long it = cursor;
       cursor += gridDim.x;
       if (it >= total_items) {
-        item_of[st] = -1;
+        item_of[st].x = -1;
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
         return false;
       }
@@ -243,7 +247,8 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
       if (i < n_filled[b] || i >= L) continue;       // not an active mask row
       const int base = chunk * kStreamChunk;
       const uint32_t bytes = (uint32_t)min(kStreamChunk, V - base) * 2u;
-      item_of[st] = it;
+      item_of[st].x = row;
+      item_of[st].y = chunk;
       asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
       asm volatile(
           "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -262,7 +267,7 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
   }
   __syncthreads();
 
-  if (warp == kConfThreads / 32) {
+  if (warp == kStreamThreads / 32) {
     // ---- producer warp: fill the ring, then refill each stage as soon as the consumers release it
     if (lane == 0) {
       bool more = true;
@@ -278,21 +283,20 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
   for (uint32_t n = 0;; ++n) {
     const int st = n & (kStreamStages - 1);
     if (!cs_mbar_wait(cs_smem_u32(full + st), (n / kStreamStages) & 1u)) return;   // bounded; never expected
-    const long long it = item_of[st];
-    if (it < 0) break;
-    const int row = (int)(it / n_chunks), chunk = (int)(it - (long long)row * n_chunks);
+    const int row = item_of[st].x, chunk = item_of[st].y;
+    if (row < 0) break;
     const int base = chunk * kStreamChunk;
     const uint4* src = reinterpret_cast<const uint4*>(stage_mem + (size_t)st * kStreamChunk * 2);
-    uint32_t w[kConfVecs * 4];
+    uint32_t w[kStreamVecs * 4];
 #pragma unroll
-    for (int k = 0; k < kConfVecs; ++k) {
-      const uint4 v = src[k * kConfThreads + tid];
+    for (int k = 0; k < kStreamVecs; ++k) {
+      const uint4 v = src[k * kStreamThreads + tid];
       w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
     }
     if (base + kStreamChunk > V) {                   // last chunk of a row: words past the row end act as padding
 #pragma unroll
-      for (int i = 0; i < kConfVecs * 4; ++i) {
-        const int e0 = base + ((i >> 2) * kConfThreads + tid) * 8 + (i & 3) * 2;
+      for (int i = 0; i < kStreamVecs * 4; ++i) {
+        const int e0 = base + ((i >> 2) * kStreamThreads + tid) * 8 + (i & 3) * 2;
         if (e0 >= V) w[i] = 0xF149F149u;
       }
     }
@@ -304,7 +308,7 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
       mx[q] = w[q];
     }
 #pragma unroll
-    for (int i = 4; i < kConfVecs * 4; ++i) {
+    for (int i = 4; i < kStreamVecs * 4; ++i) {
       w[i] = bf162_max(w[i], 0xF149F149u);
       mx[i & 3] = bf162_max(mx[i & 3], w[i]);
     }
@@ -319,12 +323,12 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
     if (tid == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(cs_smem_u32(empty + st)) : "memory");
     m = fm[0];
 #pragma unroll
-    for (int q = 1; q < kConfThreads / 32; ++q) m = fmaxf(m, fm[q]);
+    for (int q = 1; q < kStreamThreads / 32; ++q) m = fmaxf(m, fm[q]);
     if (m_thread == m) {                             // lowest index attaining the maximum (descending scan)
       int a = 0x7fffffff;
 #pragma unroll
-      for (int i = kConfVecs * 4 - 1; i >= 0; --i) {
-        const int e0 = base + ((i >> 2) * kConfThreads + tid) * 8 + (i & 3) * 2;
+      for (int i = kStreamVecs * 4 - 1; i >= 0; --i) {
+        const int e0 = base + ((i >> 2) * kStreamThreads + tid) * 8 + (i & 3) * 2;
         if (__uint_as_float(w[i] & 0xffff0000u) == m) a = e0 + 1;
         if (__uint_as_float(w[i] << 16) == m) a = e0;
       }
@@ -335,7 +339,7 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
     const unsigned long long L2 = pack2(kLog2e, kLog2e), NM = pack2(-m * kLog2e, -m * kLog2e);
     unsigned long long sA = pack2(0.f, 0.f), sB = sA, tA = sA, tB = sA;
 #pragma unroll
-    for (int i = 0; i < kConfVecs * 4; i += 2) {
+    for (int i = 0; i < kStreamVecs * 4; i += 2) {
       const unsigned long long dA = fma2(pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u)), L2, NM);
       const unsigned long long dB = fma2(pack2(__uint_as_float(w[i + 1] << 16), __uint_as_float(w[i + 1] & 0xffff0000u)), L2, NM);
       float a0, a1, b0, b1;
@@ -362,7 +366,7 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
     if (tid == 0) {
       float ss = 0.f, tt = 0.f;
 #pragma unroll
-      for (int q = 0; q < kConfThreads / 32; ++q) { ss += fs[q]; tt += ft[q]; }
+      for (int q = 0; q < kStreamThreads / 32; ++q) { ss += fs[q]; tt += ft[q]; }
       part[(size_t)row * n_chunks + chunk] = make_float4(m, ss, tt, __int_as_float(fa));
     }
   }
@@ -577,9 +581,9 @@ int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* log
         return WEDLM_ERR_CUDA;
       int dev = 0, sms = 148;
       if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-      long long grid = (long long)sms * 3;                       // three 64 KB rings per SM
+      long long grid = (long long)sms * kStreamBlocksPerSM;
       if (grid > blocks) grid = blocks;
-      conf_stream_kernel<<<(unsigned)grid, kConfThreads + 32, smem, st>>>(s.W, s.V, n_chunks, blocks, (const T*)logits, n_filled,
+      conf_stream_kernel<<<(unsigned)grid, kStreamThreads + 32, smem, st>>>(s.W, s.V, n_chunks, blocks, (const T*)logits, n_filled,
                                                                       window_len, part);
     } else {
       conf_partial_kernel<T, false><<<(unsigned)blocks, kConfThreads, 0, st>>>(s.W, s.V, n_chunks, (const T*)logits, n_filled, window_len, part);
