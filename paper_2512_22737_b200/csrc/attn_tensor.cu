@@ -8,7 +8,7 @@
 // rotated K and V were staged there by the RoPE/stage kernel before this kernel starts.
 //
 // One CTA = one (b, g, 128-row tile, key chunk).  Warps 0-3 (128 threads, one query row each) run the
-// online softmax; warp 4 lane 0 issues every MMA; warp 5 lane 0 issues every TMA copy.  Per 64-key tile:
+// online softmax; warp 4 lane 0 issues every MMA; warps 5 and 6 issue the TMA copies of K and V.  Per 64-key tile:
 //     S[t&1] = Q K_t^T   (tcgen05.mma, 8 k-steps, fp32 in TMEM columns 0..127, double buffered)
 //     softmax threads: tcgen05.ld S row -> mask -> running max (lazy rescale) -> p = 2^(s*c - m*c)
 //                      -> bf16 P tile into shared memory (128-byte swizzle)
@@ -29,7 +29,7 @@ constexpr int kTileN = 64;            // keys per tile (4 pages)
 constexpr int kD = 128;               // head size
 constexpr int kPage = 16;
 static_assert(kTileN == 4 * kPage, "a tile is four pages");
-constexpr int kThreadsT = 192;        // 4 softmax warps + MMA issue warp + TMA producer warp
+constexpr int kThreadsT = 224;        // 4 softmax warps + MMA issue warp + two TMA producer warps
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kLazyRescaleLog2 = 8.0f;   // keep the old reference while the max grew by < 2^8
 
@@ -62,7 +62,7 @@ struct TensorAttnParams {
 
 #ifdef WEDLM_ATTN_TRACE
 // Debug builds only: per-tile timestamps of one CTA, [role][tile][event].
-__device__ long long g_attn_trace[3 * 256 * 8];
+__device__ long long g_attn_trace[4 * 256 * 8];
 #define TRACE(role, t, ev) do { if (trace_on && (unsigned)(t) < 256u) g_attn_trace[((role) * 256 + (t)) * 8 + (ev)] = clock64(); } while (0)
 #else
 #define TRACE(role, t, ev) do { } while (0)
@@ -303,10 +303,12 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         if (p.status) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
       }
     }
-  } else if (warp == 5) {
-    // ------------------------------------------------------------------ TMA producer warp
-    // A tile is 8 copies of 2 KB (4 pages x 2 column halves).  Lanes 0..7 each look up their page and
-    // issue their copy, so that the 8 copies of a tile leave in one warp instruction.
+  } else if (warp >= 5) {
+    // ------------------------------------------------------------------ TMA producer warps
+    // Warp 5 streams the K tiles (and loads Q), warp 6 the V tiles; each refills a stage as soon as the
+    // MMAs that read it have completed.  A tile is 8 copies of 2 KB (4 pages x 2 column halves): lanes
+    // 0..7 each look up their page and issue their copy, so a tile leaves in one warp instruction.
+    const bool is_k = (warp == 5);
     bool ok = true;
     const int oob_row = p.num_pages * p.Hkv * kPage;        // a row coordinate past the end: zero fill
     const int pg = (lane >> 1) & 3, half = lane & 1;
@@ -318,51 +320,39 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       int pp = -1;
       if (lp < p.max_pages) pp = p.block_table[(size_t)b * p.max_pages + lp];
       if (pp < 0 || pp >= p.num_pages) {
-        if (key0 < kv_end && p.status) atomicOr(p.status, lp < p.max_pages ? WEDLM_STATUS_BAD_PAGE : WEDLM_STATUS_BAD_LENGTH);
+        if (is_k && key0 < kv_end && p.status) atomicOr(p.status, lp < p.max_pages ? WEDLM_STATUS_BAD_PAGE : WEDLM_STATUS_BAD_LENGTH);
         return oob_row;
       }
       return (pp * p.Hkv + g) * kPage;
-    };
-    auto load_tile = [&](const CUtensorMap* map, uint32_t dst_stage, uint32_t full_bar, int y) {
-      if (lane == 0) mbar_expect_tx(full_bar, kStageBytes);
-      __syncwarp();
-      if (lane < 8) tma_load_2d(dst_stage + lane_dst, map, half * 64, y, full_bar);
     };
     auto wait_all = [&](uint32_t barrier, uint32_t parity) -> bool {      // lane 0 waits, the warp follows
       int good = 1;
       if (lane == 0) good = mbar_wait(barrier, parity) ? 1 : 0;
       return __shfl_sync(0xffffffffu, good, 0) != 0;
     };
-    if (lane == 0) {
+    if (is_k && lane == 0) {
       // Q tile: two 64-element halves of [W_t slots x G heads] rows
       const int q_slots = min(p.W_t, p.W);        // box height along the window dimension
       mbar_expect_tx(bar(Q_FULL), (uint32_t)(2 * 64 * p.G * q_slots * 2));
       tma_load_4d(sbase + kOffQ, &tm_q, 0, g * p.G, slot0, b, bar(Q_FULL));
       tma_load_4d(sbase + kOffQ + kHalfQ, &tm_q, 64, g * p.G, slot0, b, bar(Q_FULL));
     }
-    // order of issue follows the order in which stages come free: K_{u+1} (after Q K_{u-1}^T), then
-    // V_u (after P V_{u-2})
-    int y_cur = page_row(0);
-    load_tile(&tm_k, sbase + kOffK, bar(K_FULL0), y_cur);
-    int y_next = (1 < T) ? page_row(1) : oob_row;
-    for (int u = 0; ok && u < T; ++u) {
-      if (u + 1 < T) {
-        const uint32_t st1 = (uint32_t)(u + 1) & 1u;
-        TRACE(1, u, 0);
-        if (u + 1 >= 2) ok = wait_all(bar(K_FREE0 + st1), ((uint32_t)(u - 1) >> 1) & 1u);
-        if (!ok) break;
-        TRACE(1, u, 2);
-        load_tile(&tm_k, sbase + kOffK + st1 * kStageBytes, bar(K_FULL0 + st1), y_next);
-        TRACE(1, u, 3);
-      }
-      const uint32_t st = (uint32_t)u & 1u;
-      if (u >= 2) ok = wait_all(bar(V_FREE0 + st), ((uint32_t)(u - 2) >> 1) & 1u);
+    const CUtensorMap* map = is_k ? &tm_k : &tm_v;
+    const uint32_t stage0 = sbase + (is_k ? kOffK : kOffV);
+    const int full0 = is_k ? K_FULL0 : V_FULL0, free0 = is_k ? K_FREE0 : V_FREE0;
+    int y_next = page_row(0);
+    for (int t = 0; ok && t < T; ++t) {
+      const uint32_t st = (uint32_t)t & 1u;
+      const int y = y_next;
+      if (t + 1 < T) y_next = page_row(t + 1);              // table entry of the next tile, used one iteration later
+      TRACE(is_k ? 1 : 3, t, 0);
+      if (t >= 2) ok = wait_all(bar(free0 + st), ((uint32_t)(t - 2) >> 1) & 1u);
       if (!ok) break;
-      TRACE(1, u, 4);
-      load_tile(&tm_v, sbase + kOffV + st * kStageBytes, bar(V_FULL0 + st), y_cur);
-      TRACE(1, u, 5);
-      y_cur = y_next;
-      if (u + 2 < T) y_next = page_row(u + 2);      // consumed one iteration later
+      TRACE(is_k ? 1 : 3, t, 1);
+      if (lane == 0) mbar_expect_tx(bar(full0 + st), kStageBytes);
+      __syncwarp();
+      if (lane < 8) tma_load_2d(stage0 + st * kStageBytes + lane_dst, map, half * 64, y, bar(full0 + st));
+      TRACE(is_k ? 1 : 3, t, 2);
     }
     if (!ok && lane == 0) {
       *abort_flag = 1;
@@ -554,7 +544,7 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
 
 #ifdef WEDLM_ATTN_TRACE
 extern "C" int wedlm_debug_read_attn_trace(long long* host_dst) {
-  return cudaMemcpyFromSymbol(host_dst, g_attn_trace, sizeof(long long) * 3 * 256 * 8) == cudaSuccess ? 0 : -4;
+  return cudaMemcpyFromSymbol(host_dst, g_attn_trace, sizeof(long long) * 4 * 256 * 8) == cudaSuccess ? 0 : -4;
 }
 #endif
 
