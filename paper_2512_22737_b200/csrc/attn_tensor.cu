@@ -170,6 +170,29 @@ __device__ __forceinline__ float ex2_approx(float x) {      // 2^x on the SFU; f
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Packed fp32x2 arithmetic of sm_100 (two lanes per instruction) and the 3-input maximum.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {     // a register pair, no instruction
+  return ((unsigned long long)__float_as_uint(hi) << 32) | (unsigned long long)__float_as_uint(lo);
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+  lo = __uint_as_float((unsigned)(v & 0xffffffffull));
+  hi = __uint_as_float((unsigned)(v >> 32));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -381,29 +404,27 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tmem_wait_ld();
       }
       TRACE(2, t, 2);
-      float s[64];
       const int tile0 = kv_begin + t * kTileN;
       const bool need_mask = tile0 + kTileN > min(P + slot0 + 1, kv_end);   // block-uniform
-      float m_tile = -CUDART_INF_F;
+      float m_tile;
       if (need_mask) {
+        m_tile = -CUDART_INF_F;
 #pragma unroll
         for (int cc = 0; cc < 64; ++cc) {
           const int key = tile0 + cc;
           float x = __uint_as_float(raw[cc]);
           x = (key <= limit && key < kv_end) ? x : -CUDART_INF_F;
-          s[cc] = x;
+          raw[cc] = __float_as_uint(x);
           m_tile = fmaxf(m_tile, x);
         }
       } else {
         float m4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
         for (int cc = 0; cc < 64; cc += 8) {
-#pragma unroll
-          for (int e = 0; e < 8; ++e) s[cc + e] = __uint_as_float(raw[cc + e]);
-          m4[0] = fmaxf(m4[0], fmaxf(s[cc + 0], s[cc + 1]));
-          m4[1] = fmaxf(m4[1], fmaxf(s[cc + 2], s[cc + 3]));
-          m4[2] = fmaxf(m4[2], fmaxf(s[cc + 4], s[cc + 5]));
-          m4[3] = fmaxf(m4[3], fmaxf(s[cc + 6], s[cc + 7]));
+          m4[0] = max3(m4[0], __uint_as_float(raw[cc + 0]), __uint_as_float(raw[cc + 1]));
+          m4[1] = max3(m4[1], __uint_as_float(raw[cc + 2]), __uint_as_float(raw[cc + 3]));
+          m4[2] = max3(m4[2], __uint_as_float(raw[cc + 4]), __uint_as_float(raw[cc + 5]));
+          m4[3] = max3(m4[3], __uint_as_float(raw[cc + 6]), __uint_as_float(raw[cc + 7]));
         }
         m_tile = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
       }
@@ -416,14 +437,27 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         moved = true;
       }
       const float neg_mc = (m_ref == -CUDART_INF_F) ? 0.f : -m_ref * c;
-      float sum = 0.f, sum2 = 0.f;
+      // p = 2^(s*c - m*c): the scale and the reference are folded into one packed FMA per two scores
+      const unsigned long long C2 = pack2(c, c), NM2 = pack2(neg_mc, neg_mc);
+      unsigned long long sumA = pack2(0.f, 0.f), sumB = sumA;
       uint32_t pk[32];
 #pragma unroll
-      for (int cc = 0; cc < 64; cc += 2) {
-        const float p0 = ex2_approx(fmaf(s[cc], c, neg_mc));
-        const float p1 = ex2_approx(fmaf(s[cc + 1], c, neg_mc));
-        if ((cc & 2) == 0) sum += p0 + p1; else sum2 += p0 + p1;
+      for (int cc = 0; cc < 64; cc += 4) {
+        float a0, a1, b0, b1;
+        unpack2(fma2(pack2(__uint_as_float(raw[cc]), __uint_as_float(raw[cc + 1])), C2, NM2), a0, a1);
+        unpack2(fma2(pack2(__uint_as_float(raw[cc + 2]), __uint_as_float(raw[cc + 3])), C2, NM2), b0, b1);
+        const float p0 = ex2_approx(a0), p1 = ex2_approx(a1), p2 = ex2_approx(b0), p3 = ex2_approx(b1);
+        sumA = add2(sumA, pack2(p0, p1));
+        sumB = add2(sumB, pack2(p2, p3));
         pk[cc >> 1] = pack_bf16(p0, p1);
+        pk[(cc >> 1) + 1] = pack_bf16(p2, p3);
+      }
+      float sum, sum2;
+      {
+        float x0, x1;
+        unpack2(add2(sumA, sumB), x0, x1);
+        sum = x0;
+        sum2 = x1;
       }
       l = l * alpha + (sum + sum2);
       // P buffer and O are free / stable once P V_{t-1} has completed
