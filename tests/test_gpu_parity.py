@@ -72,6 +72,28 @@ def test_head_geometries(impl, Hq, Hkv, D):
     pu.full_parity(cfg, make_step(cfg, seed=Hq * 7 + D), attn_impl="generic")
 
 
+@pytest.mark.parametrize("Hq,Hkv,W", [(8, 8, 40), (8, 4, 70), (16, 2, 20), (16, 1, 9), (4, 4, 130)])
+def test_tensor_path_group_sizes(Hq, Hkv, W):
+    """G = 1, 2, 8, 16 with D = 128: the 128-row tile holds 128/G window slots; windows that need one,
+    two (partial) or more row tiles."""
+    import parity_util as pu
+    cfg = _small_qwen(batch=2, window=W, n_q_heads=Hq, n_kv_heads=Hkv, prefix_lo=200, prefix_hi=400, vocab=2048,
+                      name="groups")
+    inp = make_step(cfg, seed=Hq * 100 + Hkv)
+    r = pu.full_parity(cfg, inp, attn_impl="tensor")
+    assert r["attn_err"] <= pu.ATTN_REL_TOL
+
+
+@pytest.mark.parametrize("W", [128, 1024])
+def test_large_windows(W):
+    """Window sizes up to the maximum the ABI accepts (generic path at 1024, both paths at 128)."""
+    import parity_util as pu
+    cfg = _small_qwen(batch=1, window=W, n_q_heads=4, n_kv_heads=1, prefix_lo=50, prefix_hi=50, vocab=512,
+                      name="bigwindow")
+    inp = make_step(cfg, seed=W)
+    pu.full_parity(cfg, inp, attn_impl="generic" if W > 128 else "tensor")
+
+
 @pytest.mark.parametrize("P", [0, 1, 15, 16, 17, 31, 33])
 def test_page_boundaries(P):
     import parity_util as pu
