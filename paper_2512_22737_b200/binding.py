@@ -305,6 +305,18 @@ class DecodeStep:
                                 self.lse, self.committed_tokens, self.committed_count, self.filled_count,
                                 self.conf_ws)
 
+    def capture_graph(self, d: Dict[str, torch.Tensor], window_len=None, remaining_budget=None) -> "torch.cuda.CUDAGraph":
+        """Capture reorder -> attention -> confidence/commit on these fixed buffers into a CUDA graph.
+        The calls are asynchronous and read their sizes from device memory, so one capture serves
+        every later step: replaying it advances the device-resident window state again.  One
+        un-captured run comes first (it performs the per-device set-up)."""
+        self.run(d, window_len, remaining_budget)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.run(d, window_len, remaining_budget)
+        return graph
+
     def run(self, d: Dict[str, torch.Tensor], window_len=None, remaining_budget=None) -> None:
         """d holds device tensors named as in workloads.make_step(); window state is updated in place."""
         self.reorder(d["filled"], d["window_tokens"], d["prefix_len"], window_len)

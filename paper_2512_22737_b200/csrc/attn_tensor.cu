@@ -629,9 +629,17 @@ int launch_attn_tensor(const Shape& s, const AttnPlan& plan, const void* q_rot, 
   p.block_table = block_table; p.prefix_len = prefix_len; p.order = order;
   p.out = (__nv_bfloat16*)out; p.part_o = part_o; p.part_ml = part_ml; p.status = status;
 
-  // per device; cheap enough to repeat on every launch
-  if (cudaFuncSetAttribute(attn_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
-    return WEDLM_ERR_CUDA;
+  // the opt-in to large dynamic shared memory is per device: done once for each device ordinal
+  {
+    static bool attr_done[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return WEDLM_ERR_CUDA;
+    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+      if (cudaFuncSetAttribute(attn_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
+        return WEDLM_ERR_CUDA;
+      if (dev >= 0 && dev < 64) attr_done[dev] = true;
+    }
+  }
   dim3 grid(plan.n_splits * n_mtiles, s.Hkv, s.B);
   attn_tensor_kernel<<<grid, kThreadsT, kSmemBytes, st>>>(tm_q, tm_k, tm_v, p);
   count_launch();

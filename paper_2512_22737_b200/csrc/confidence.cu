@@ -577,10 +577,18 @@ int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* log
     const bool vec = (s.V % VecTraits<T>::VL == 0) && ((uintptr_t)logits % 16 == 0);
     if (vec) {
       const size_t smem = (size_t)kStreamStages * kStreamChunk * 2 + kStreamStages * 24;
-      if (cudaFuncSetAttribute(conf_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return WEDLM_ERR_CUDA;
+      static bool attr_done[64] = {};
+      static int sm_count[64] = {};
       int dev = 0, sms = 148;
-      if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+      if (cudaGetDevice(&dev) != cudaSuccess) return WEDLM_ERR_CUDA;
+      if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+        if (cudaFuncSetAttribute(conf_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+          return WEDLM_ERR_CUDA;
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (dev >= 0 && dev < 64) { attr_done[dev] = true; sm_count[dev] = sms; }
+      } else {
+        sms = sm_count[dev];
+      }
       long long grid = (long long)sms * kStreamBlocksPerSM;
       if (grid > blocks) grid = blocks;
       conf_stream_kernel<<<(unsigned)grid, kStreamThreads + 32, smem, st>>>(s.W, s.V, n_chunks, blocks, (const T*)logits, n_filled,

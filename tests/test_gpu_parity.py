@@ -294,3 +294,33 @@ def test_cfg3_batched_serving_full_size_sampled(impl):
 @pytest.mark.parametrize("impl", IMPLS)
 def test_cfg4_long_context_full_size_sampled(impl):
     _sampled_full_size("cfg4_long", impl)
+
+
+def test_step_is_capturable_in_a_cuda_graph_and_replays_identically():
+    """The three calls use only the caller's stream and device-resident sizes: a captured step replayed
+    on restored inputs reproduces the eager results bit for bit."""
+    import paper_2512_22737_b200 as w
+    import parity_util as pu
+    cfg = _small_qwen(batch=3, window=16, prefix_lo=100, prefix_hi=900, vocab=8192, boost=14.0, name="graph")
+    inp = make_step(cfg, seed=123)
+    d = pu.device_inputs(inp)
+    c = w.config_for(cfg, max_pages_per_seq=inp["block_table"].shape[1], num_pages=inp["k_cache"].shape[0],
+                     max_prefix_len=int(inp["prefix_len"].max()))
+    step = w.DecodeStep(c)
+    state0 = {k: d[k].clone() for k in ("filled", "window_tokens", "prefix_len")}
+    step.run(d)
+    torch.cuda.synchronize()
+    eager = {k: getattr(step, k).clone() for k in ("out", "argmax", "entropy", "committed_count", "committed_tokens")}
+    eager_state = {k: d[k].clone() for k in state0}
+    for k, v in state0.items():
+        d[k].copy_(v)
+    graph = step.capture_graph(d)          # runs once eagerly, then captures once
+    for _ in range(2):
+        for k, v in state0.items():
+            d[k].copy_(v)
+        graph.replay()
+        torch.cuda.synchronize()
+        for k, v in eager.items():
+            assert torch.equal(getattr(step, k).view(torch.uint8), v.view(torch.uint8)), k
+        for k, v in eager_state.items():
+            assert torch.equal(d[k], v), k
