@@ -99,7 +99,12 @@ int wedlm_version(void);
  *   the two CUDA events (cudaEvent_t cast to void*, host handles, either may be NULL) on its stream
  *   immediately before and after its main attention kernel, so that the kernel can be timed inside
  *   a longer sequence of launches.  One-shot: the hook is cleared by that call. */
+/* wedlm_selftest_wait_expiry: launches one small CTA that waits, with at most max_polls (1..2^24) polls,
+ *   on an on-chip barrier that nothing ever signals - the situation the bounded waits of the tensor-core
+ *   attention kernel exist for.  The kernel gives up, ORs WEDLM_STATUS_WAIT_EXPIRED into *status (device
+ *   i32, required) and returns normally; the context stays usable. */
 unsigned long long wedlm_launch_count(void);
+int wedlm_selftest_wait_expiry(uint32_t max_polls, int32_t* status, void* stream);
 int wedlm_profile_next_attn(void* event_before, void* event_after);
 
 /*

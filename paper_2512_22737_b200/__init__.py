@@ -21,6 +21,7 @@ from .binding import (  # noqa: F401
     wedlm_launch_count,
     wedlm_profile_next_attn,
     wedlm_reorder,
+    wedlm_selftest_wait_expiry,
     wedlm_strerror,
     wedlm_version,
     wedlm_window_attn,

@@ -72,6 +72,8 @@ def load_library() -> ctypes.CDLL:
     lib.wedlm_launch_count.argtypes = []
     lib.wedlm_profile_next_attn.restype = ctypes.c_int
     lib.wedlm_profile_next_attn.argtypes = [vp, vp]
+    lib.wedlm_selftest_wait_expiry.restype = ctypes.c_int
+    lib.wedlm_selftest_wait_expiry.argtypes = [ctypes.c_uint32, i32p, vp]
     lib.wedlm_reorder.restype = ctypes.c_int
     lib.wedlm_reorder.argtypes = [cfgp, u8p, i32p, i32p, i32p, i32p, i32p, i32p, i32p, i32p, i32p, vp]
     lib.wedlm_window_attn_workspace_bytes.restype = ctypes.c_size_t
@@ -119,6 +121,11 @@ def wedlm_profile_next_attn(event_before: Optional[torch.cuda.Event], event_afte
         return ctypes.c_void_p(ev.cuda_event)
     _check(load_library().wedlm_profile_next_attn(handle(event_before), handle(event_after)),
            "wedlm_profile_next_attn")
+
+
+def wedlm_selftest_wait_expiry(max_polls: int, status: torch.Tensor, stream=None) -> None:
+    _check(load_library().wedlm_selftest_wait_expiry(ctypes.c_uint32(max_polls), _ptr(status, torch.int32, "status"),
+                                                     _stream(stream)), "wedlm_selftest_wait_expiry")
 
 
 def make_config(*, batch, window, n_q_heads=1, n_kv_heads=1, head_dim=128, page_size=16,

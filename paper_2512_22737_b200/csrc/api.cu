@@ -140,6 +140,11 @@ int wedlm_version(void) { return 100; }
 
 unsigned long long wedlm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
+int wedlm_selftest_wait_expiry(uint32_t max_polls, int32_t* status, void* stream) {
+  if (status == nullptr || max_polls == 0 || max_polls > (1u << 24)) return WEDLM_ERR_INVALID_ARG;
+  return launch_wait_expiry_selftest(max_polls, status, (cudaStream_t)stream);
+}
+
 int wedlm_profile_next_attn(void* event_before, void* event_after) {
   t_ev_before = (cudaEvent_t)event_before;
   t_ev_after = (cudaEvent_t)event_after;

@@ -574,13 +574,41 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
   return fn;
 }
 
+// Self-test of the bounded-wait mechanism: one CTA waits on an mbarrier that nothing ever arrives at,
+// with the same polling helper as the attention kernel but a caller-chosen limit, then reports the
+// expiry through the status word and returns normally.
+__global__ void wait_expiry_selftest_kernel(uint32_t max_polls, int32_t* status) {
+  __shared__ uint64_t never;
+  const uint32_t bar = smem_u32(&never);
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    bool done = false;
+    for (uint32_t it = 0; it < max_polls && !done; ++it) done = mbar_try_wait(bar, 0);
+    if (!done && status) atomicOr(status, WEDLM_STATUS_WAIT_EXPIRED);
+  }
+}
+
 }  // namespace
+
+int launch_wait_expiry_selftest(uint32_t max_polls, int32_t* status, cudaStream_t st) {
+  wait_expiry_selftest_kernel<<<1, 32, 0, st>>>(max_polls, status);
+  count_launch();
+  return cuda_ok(cudaGetLastError());
+}
+
+namespace {
 
 #ifdef WEDLM_ATTN_TRACE
 extern "C" int wedlm_debug_read_attn_trace(long long* host_dst) {
   return cudaMemcpyFromSymbol(host_dst, g_attn_trace, sizeof(long long) * 4 * 256 * 8) == cudaSuccess ? 0 : -4;
 }
 #endif
+
+}  // namespace
 
 bool attn_tensor_supported(const wedlm_config_t* c) {
   if (c->dtype != WEDLM_DTYPE_BF16 || c->head_dim != kD || c->page_size != kPage) return false;

@@ -72,6 +72,8 @@ int launch_attn_tensor(const Shape& s, const AttnPlan& plan, const void* q_rot, 
                        const int32_t* order, void* out, float* part_o, float* part_ml, int32_t* status,
                        cudaStream_t st);
 
+int launch_wait_expiry_selftest(uint32_t max_polls, int32_t* status, cudaStream_t st);
+
 int launch_attn_merge(const Shape& s, const AttnPlan& plan, const int32_t* prefix_len, const float* part_o,
                       const float* part_ml, void* out, cudaStream_t st);
 

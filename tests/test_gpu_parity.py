@@ -324,3 +324,17 @@ def test_step_is_capturable_in_a_cuda_graph_and_replays_identically():
             assert torch.equal(getattr(step, k).view(torch.uint8), v.view(torch.uint8)), k
         for k, v in eager_state.items():
             assert torch.equal(d[k], v), k
+
+
+def test_a_wait_that_nothing_satisfies_expires_and_reports_status():
+    """Failure detection without a fault: the wait gives up after its poll limit, the status word
+    carries WEDLM_STATUS_WAIT_EXPIRED, and the context keeps working."""
+    import paper_2512_22737_b200 as w
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    w.wedlm_selftest_wait_expiry(20000, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == w.binding.WEDLM_STATUS_WAIT_EXPIRED
+    # the context is intact: a normal step still runs and matches the oracle
+    import parity_util as pu
+    cfg = _small_qwen(batch=1, window=8, prefix_lo=40, prefix_hi=40, vocab=1024, name="afterwait")
+    pu.full_parity(cfg, make_step(cfg, seed=2))
