@@ -536,10 +536,11 @@ def run_loop(args):
     pt = make_prompts_and_targets(m, B, P, N)
     results = []
     lse0 = None
-    for W in args.loop_windows:
+    runs = [(W, "streaming") for W in args.loop_windows] + [(W, "block") for W in args.loop_block_windows]
+    for W, mode in runs:
         for tilt_name, tilt in args.loop_tilts:
             dec = StreamingDecoder(m, {}, batch=B, window=W, max_total_len=P + N, tau=0.3, lam=0.1, tilt=0.0,
-                                   target=pt["target"])
+                                   target=pt["target"], commit_mode=mode)
             dec.wt = wts
             dec.prefill(pt["prompt"])
             if lse0 is None:                    # log-sum-exp of the untilted logits, measured once
@@ -554,7 +555,7 @@ def run_loop(args):
             dt = time.perf_counter() - t0
             n_gen = sum(len(y) for y in out["y"])
             on_target = sum(int(out["y"][bb] == pt["target"][bb, P:P + N].tolist()) for bb in range(B))
-            results.append({"window": W, "tilt": f"{tilt_name}+{tilt:g}", "tokens_per_s": n_gen / dt, "seconds": dt,
+            results.append({"window": W, "commit": mode, "tilt": f"{tilt_name}+{tilt:g}", "tokens_per_s": n_gen / dt, "seconds": dt,
                             "steps": out["steps"], "tokens_per_step_per_seq": n_gen / B / max(out["steps"], 1),
                             "p_cache": out["p_cache"], "sequences_equal_to_target": on_target})
             log(results[-1])
@@ -584,6 +585,8 @@ def main():
     ap.add_argument("--loop-batch", type=int, default=16)
     ap.add_argument("--loop-new-tokens", type=int, default=1024)
     ap.add_argument("--loop-windows", type=lambda s: [int(x) for x in s.split(",")], default=[16, 2, 1])
+    ap.add_argument("--loop-block-windows", type=lambda s: [int(x) for x in s.split(",") if x], default=[16],
+                    help="windows also run with the block-wise commit rule (the baseline of Fig. 3c)")
     ap.add_argument("--loop-tilts", type=lambda s: [(t.split(":")[0], float(t.split(":")[1])) for t in s.split(",")],
                     default=[("literal", 2.0), ("literal", 4.0), ("literal", 8.0), ("lse", 2.0), ("lse", 4.0), ("lse", 8.0)])
     args = ap.parse_args()

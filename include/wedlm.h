@@ -60,6 +60,10 @@ extern "C" {
 #define WEDLM_CONF_ENTROPY 0   /* select mask i iff  H_i + lambda * d_i <= tau   (Eq. 11) */
 #define WEDLM_CONF_MAXPROB 1   /* select mask i iff  max_v p_i(v) >= maxprob_thr          */
 
+#define WEDLM_COMMIT_STREAMING 0   /* commit the leading run of filled slots (Algorithm 1)              */
+#define WEDLM_COMMIT_BLOCK     1   /* block-wise baseline of Section 5.2 / Fig. 3c: commit nothing until  */
+                                   /* every active slot of the window is filled, then commit all of them */
+
 #define WEDLM_ATTN_AUTO    0
 #define WEDLM_ATTN_GENERIC 1   /* CUDA-core kernel, any supported shape, bf16 or fp32     */
 #define WEDLM_ATTN_TENSOR  2   /* tcgen05 + TMA kernel, bf16, head_dim 128, page 16       */
@@ -85,6 +89,7 @@ typedef struct wedlm_config {
   int32_t mask_token_id;      /* token id written into fresh mask slots                    */
   int32_t max_prefix_len;     /* host-known upper bound of prefix_len[b]; sizes the grid   */
   int32_t attn_impl;          /* WEDLM_ATTN_*                                              */
+  int32_t commit_mode;        /* WEDLM_COMMIT_*                                            */
 } wedlm_config_t;
 
 /* Human-readable text of a return code.  Host pointer to a static string. */
@@ -120,6 +125,7 @@ int wedlm_profile_next_attn(void* event_before, void* event_after);
  *   tokens_phys   out i32 [B,W]  window_tokens[perm[i]], or NULL
  *   n_filled      out i32 [B]    number of filled active slots (= first mask's physical row)
  *   n_commit      out i32 [B]    length of the leading run of filled slots in logical order
+ *                                (WEDLM_COMMIT_BLOCK: window_len if every active slot is filled, else 0)
  */
 int wedlm_reorder(const wedlm_config_t* cfg, const uint8_t* filled, const int32_t* window_tokens,
                   const int32_t* prefix_len, const int32_t* window_len,

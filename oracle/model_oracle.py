@@ -70,7 +70,8 @@ def forward_window(weights: Dict[str, np.ndarray], mcfg, committed: Sequence[int
 
 
 def decode(weights, mcfg, prompt: Sequence[int], target: Sequence[int], *, tilt: float, window: int,
-           max_new_tokens: int, conf_mode: str, tau: float, lam: float, maxprob_thr: float) -> Dict[str, object]:
+           max_new_tokens: int, conf_mode: str, tau: float, lam: float, maxprob_thr: float,
+           block_commit: bool = False) -> Dict[str, object]:
     """Algorithm 1 for one sequence on the model above; logits[row, target[position of row]] += tilt."""
     prompt = [int(t) for t in prompt]
 
@@ -83,4 +84,4 @@ def decode(weights, mcfg, prompt: Sequence[int], target: Sequence[int], *, tilt:
 
     return orc.decode_loop(forward, prefix_len=len(prompt), window=window, max_new_tokens=max_new_tokens,
                            conf_mode=conf_mode, tau=tau, lam=lam, maxprob_thr=maxprob_thr,
-                           mask_token_id=mcfg.mask_token_id)
+                           mask_token_id=mcfg.mask_token_id, block_commit=block_commit)

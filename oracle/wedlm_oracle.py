@@ -63,7 +63,7 @@ def round_to_bf16(x: np.ndarray) -> np.ndarray:
 # Topological Reordering (Eq. 5-6) and the commit length (Algorithm 1, Commit)
 # ----------------------------------------------------------------------------------------
 def reorder(filled: np.ndarray, prefix_len: np.ndarray,
-            window_len: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+            window_len: Optional[np.ndarray] = None, block_commit: bool = False) -> Dict[str, np.ndarray]:
     """Stable partition of each window: filled slots (ascending logical index) first, then masks
     (ascending).  pos_ids keeps each slot's logical position P + j.  Slots at or beyond
     window_len (a window that shrank at the end of generation) are treated as trailing masks.
@@ -87,7 +87,11 @@ def reorder(filled: np.ndarray, prefix_len: np.ndarray,
             inv[b, j] = i
             pos[b, i] = int(prefix_len[b]) + j
         n_filled[b] = len(observed)
-        n_commit[b] = masked[0] if masked else W
+        if block_commit:
+            # block-wise baseline (Section 5.2, Fig. 2): nothing is committed until the whole block is final
+            n_commit[b] = L if (len(observed) == L and L > 0) else 0
+        else:
+            n_commit[b] = masked[0] if masked else W
     return dict(perm=perm, inv_perm=inv, pos_ids=pos, n_filled=n_filled, n_commit=n_commit)
 
 
@@ -248,7 +252,7 @@ def select_commit_refill(tokens: Sequence[int], filled: Sequence[int], window_le
                          mask_entropy: Sequence[float], mask_maxprob: Sequence[float], *,
                          conf_mode: str, tau: float, lam: float, maxprob_thr: float,
                          mask_token_id: int, remaining_budget: Optional[int] = None,
-                         fallback: bool = True) -> Dict[str, object]:
+                         fallback: bool = True, block_commit: bool = False) -> Dict[str, object]:
     """tokens/filled: the window in LOGICAL order (W slots, the first window_len active).
     mask_*[k] are the statistics of the k-th active mask in ascending logical order (that is the
     physical row n_filled + k after reordering).
@@ -264,6 +268,8 @@ def select_commit_refill(tokens: Sequence[int], filled: Sequence[int], window_le
     n = 0
     while n < L and fil[n]:
         n += 1
+    if block_commit and n < L:
+        n = 0                           # block-wise baseline: all active slots or nothing
     committed = tok[:n]
     # Masks of the current window, ascending; k-th one owns statistics row k.
     masks = [j for j in range(L) if not fil[j]]
@@ -309,11 +315,11 @@ def select_commit_refill(tokens: Sequence[int], filled: Sequence[int], window_le
 def step(inp: Dict[str, np.ndarray], *, theta: float, rope_style: int = 0, conf_mode: str,
          tau: float, lam: float, maxprob_thr: float, mask_token_id: int, page_size: int,
          window_len: Optional[np.ndarray] = None, remaining_budget: Optional[np.ndarray] = None,
-         with_attention: bool = True) -> Dict[str, object]:
+         with_attention: bool = True, block_commit: bool = False) -> Dict[str, object]:
     """All outputs of one decoding step for the arrays of workloads.make_step()."""
     filled, prefix_len = inp["filled"], inp["prefix_len"]
     B, W = filled.shape
-    ro = reorder(filled, prefix_len, window_len)
+    ro = reorder(filled, prefix_len, window_len, block_commit)
     res: Dict[str, object] = dict(ro)
     res["tokens_phys"] = np.take_along_axis(np.asarray(inp["window_tokens"]), ro["perm"], axis=1)
     res["kv_slot_idx"] = stage_slots(inp["block_table"], prefix_len, W, page_size)
@@ -341,7 +347,8 @@ def step(inp: Dict[str, np.ndarray], *, theta: float, rope_style: int = 0, conf_
             argmax[b, nf:nf + n_mask], ent[b, nf:nf + n_mask], mp[b, nf:nf + n_mask],
             conf_mode=conf_mode, tau=tau, lam=lam, maxprob_thr=maxprob_thr,
             mask_token_id=mask_token_id,
-            remaining_budget=None if remaining_budget is None else int(remaining_budget[b])))
+            remaining_budget=None if remaining_budget is None else int(remaining_budget[b]),
+            block_commit=block_commit))
     res.update(argmax=argmax, entropy=ent, maxprob=mp, lse=lse, per_seq=per_seq)
     return res
 
@@ -352,7 +359,7 @@ def step(inp: Dict[str, np.ndarray], *, theta: float, rope_style: int = 0, conf_
 def decode_loop(forward: Callable[[List[int], List[int], List[int]], np.ndarray], *,
                 prefix_len: int, window: int, max_new_tokens: int, conf_mode: str, tau: float,
                 lam: float, maxprob_thr: float, mask_token_id: int,
-                max_steps: int = 100000) -> Dict[str, object]:
+                max_steps: int = 100000, block_commit: bool = False) -> Dict[str, object]:
     """Streaming Parallel Decoding (Algorithm 1) for one sequence.
 
     forward(y, tokens_phys, pos_ids) -> logits [W_len, V]: the causal forward of the reordered
@@ -377,7 +384,7 @@ def decode_loop(forward: Callable[[List[int], List[int], List[int]], np.ndarray]
         c = confidence(logits[nf:L]) if L > nf else dict(argmax=[], entropy=[], maxprob=[])
         r = select_commit_refill(tok, fil, L, P, c["argmax"], c["entropy"], c["maxprob"],
                                  conf_mode=conf_mode, tau=tau, lam=lam, maxprob_thr=maxprob_thr,
-                                 mask_token_id=mask_token_id, remaining_budget=budget)
+                                 mask_token_id=mask_token_id, remaining_budget=budget, block_commit=block_commit)
         y += r["committed_tokens"]
         trace.append(dict(window_len=L, committed=r["committed_count"], filled=r["filled_count"],
                           pos_ids=[int(p) for p in ro["pos_ids"][0][:L]]))

@@ -27,6 +27,7 @@ int check_config(const wedlm_config_t* c, bool need_cache, bool need_vocab) {
   if (c == nullptr) return WEDLM_ERR_INVALID_ARG;
   if (c->batch < 0 || c->window < 1 || c->window > 1024) return WEDLM_ERR_INVALID_ARG;
   if (c->dtype != WEDLM_DTYPE_BF16 && c->dtype != WEDLM_DTYPE_F32) return WEDLM_ERR_INVALID_ARG;
+  if (c->commit_mode != WEDLM_COMMIT_STREAMING && c->commit_mode != WEDLM_COMMIT_BLOCK) return WEDLM_ERR_INVALID_ARG;
   if (need_cache) {
     if (c->n_q_heads < 1 || c->n_kv_heads < 1 || c->n_q_heads % c->n_kv_heads != 0) return WEDLM_ERR_INVALID_ARG;
     if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128 && c->head_dim != 256) return WEDLM_ERR_UNSUPPORTED;
@@ -51,7 +52,7 @@ Shape make_shape(const wedlm_config_t* c) {
   s.B = c->batch; s.W = c->window; s.Hq = c->n_q_heads; s.Hkv = c->n_kv_heads; s.D = c->head_dim;
   s.G = c->n_kv_heads > 0 ? c->n_q_heads / c->n_kv_heads : 1;
   s.page = c->page_size; s.max_pages = c->max_pages_per_seq; s.num_pages = c->num_pages; s.V = c->vocab;
-  s.dtype = c->dtype; s.rope_style = c->rope_style; s.theta = c->rope_theta;
+  s.dtype = c->dtype; s.rope_style = c->rope_style; s.theta = c->rope_theta; s.commit_mode = c->commit_mode;
   s.scale = c->softmax_scale > 0.f ? c->softmax_scale : 1.0f / sqrtf((float)c->head_dim);
   return s;
 }

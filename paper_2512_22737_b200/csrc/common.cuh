@@ -12,7 +12,7 @@ namespace wedlm {
 struct Shape {
   int B, W, Hq, Hkv, D, G;
   int page, max_pages, num_pages, V;
-  int dtype, rope_style;
+  int dtype, rope_style, commit_mode;
   float theta, scale;
 };
 

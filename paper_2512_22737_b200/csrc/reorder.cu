@@ -6,7 +6,7 @@ namespace wedlm {
 
 // One warp per sequence.  Slot j is "observed" iff filled[j] != 0 and j < window_len.
 __global__ void __launch_bounds__(32)
-reorder_kernel(int W, const uint8_t* __restrict__ filled, const int32_t* __restrict__ window_tokens,
+reorder_kernel(int W, int commit_mode, const uint8_t* __restrict__ filled, const int32_t* __restrict__ window_tokens,
                const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ window_len,
                int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, int32_t* __restrict__ pos_ids,
                int32_t* __restrict__ tokens_phys, int32_t* __restrict__ n_filled, int32_t* __restrict__ n_commit) {
@@ -47,14 +47,15 @@ reorder_kernel(int W, const uint8_t* __restrict__ filled, const int32_t* __restr
   }
   if (lane == 0) {
     n_filled[b] = total;
-    n_commit[b] = first_mask;
+    // streaming: the leading filled run; block-wise baseline: all active slots or nothing
+    n_commit[b] = commit_mode == WEDLM_COMMIT_BLOCK ? ((total == L && L > 0) ? L : 0) : first_mask;
   }
 }
 
 int launch_reorder(const Shape& s, const uint8_t* filled, const int32_t* window_tokens, const int32_t* prefix_len,
                    const int32_t* window_len, int32_t* perm, int32_t* inv_perm, int32_t* pos_ids,
                    int32_t* tokens_phys, int32_t* n_filled, int32_t* n_commit, cudaStream_t st) {
-  reorder_kernel<<<s.B, 32, 0, st>>>(s.W, filled, window_tokens, prefix_len, window_len, perm, inv_perm, pos_ids,
+  reorder_kernel<<<s.B, 32, 0, st>>>(s.W, s.commit_mode, filled, window_tokens, prefix_len, window_len, perm, inv_perm, pos_ids,
                                      tokens_phys, n_filled, n_commit);
   count_launch();
   return cuda_ok(cudaGetLastError());

@@ -27,7 +27,7 @@ class StreamingDecoder:
     def __init__(self, mcfg, weights: Dict[str, np.ndarray], *, batch: int, window: int, max_total_len: int,
                  conf_mode: str = "entropy", tau: float = 0.3, lam: float = 0.1, maxprob_thr: float = 0.9,
                  tilt: float = 0.0, target: Optional[np.ndarray] = None, page_size: int = 16,
-                 attn_impl: str = "auto", seed: int = 0):
+                 attn_impl: str = "auto", seed: int = 0, commit_mode: str = "streaming"):
         self.m = mcfg
         self.B, self.W = batch, window
         self.dtype = torch.bfloat16 if mcfg.dtype == "bf16" else torch.float32
@@ -48,7 +48,7 @@ class StreamingDecoder:
             page_size=page_size, max_pages_per_seq=pages_per_seq, num_pages=self.num_pages, vocab=mcfg.vocab,
             dtype=mcfg.dtype, rope_theta=mcfg.rope_theta, conf_mode=conf_mode, tau=tau, lam=lam,
             maxprob_thr=maxprob_thr, mask_token_id=mcfg.mask_token_id, max_prefix_len=max_total_len,
-            attn_impl=attn_impl)
+            attn_impl=attn_impl, commit_mode=commit_mode)
         self.step_bufs = w.DecodeStep(self.cfg)
         i32 = dict(dtype=torch.int32, device="cuda")
         self.window_tokens = torch.full((batch, window), mcfg.mask_token_id, **i32)

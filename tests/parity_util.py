@@ -25,13 +25,13 @@ def bf16_from_device(t: torch.Tensor) -> np.ndarray:
     return t.detach().to(torch.float64).cpu().numpy()
 
 
-def run_gpu_step(cfg, inp, *, attn_impl="auto", window_len=None, remaining_budget=None):
+def run_gpu_step(cfg, inp, *, attn_impl="auto", window_len=None, remaining_budget=None, commit_mode="streaming"):
     """One full step on the GPU.  Returns (DecodeStep with outputs, device dict with the updated
     window state and cache)."""
     d = device_inputs(inp)
     c = w.config_for(cfg, max_pages_per_seq=inp["block_table"].shape[1], num_pages=inp["k_cache"].shape[0],
                      max_prefix_len=int(inp["prefix_len"].max()) if len(inp["prefix_len"]) else 0,
-                     attn_impl=attn_impl, batch=inp["filled"].shape[0])
+                     attn_impl=attn_impl, batch=inp["filled"].shape[0], commit_mode=commit_mode)
     step = w.DecodeStep(c)
     wl = None if window_len is None else torch.tensor(window_len, dtype=torch.int32, device="cuda")
     rb = None if remaining_budget is None else torch.tensor(remaining_budget, dtype=torch.int32, device="cuda")
@@ -42,10 +42,11 @@ def run_gpu_step(cfg, inp, *, attn_impl="auto", window_len=None, remaining_budge
     return step, d
 
 
-def oracle_step(cfg, inp, *, window_len=None, remaining_budget=None, with_attention=True):
+def oracle_step(cfg, inp, *, window_len=None, remaining_budget=None, with_attention=True, block_commit=False):
     return orc.step(inp, theta=cfg.rope_theta, conf_mode=cfg.conf_mode, tau=cfg.tau, lam=cfg.lam,
                     maxprob_thr=cfg.maxprob_thr, mask_token_id=cfg.mask_token_id, page_size=cfg.page_size,
-                    window_len=window_len, remaining_budget=remaining_budget, with_attention=with_attention)
+                    window_len=window_len, remaining_budget=remaining_budget, with_attention=with_attention,
+                    block_commit=block_commit)
 
 
 def attn_vector_error(got: np.ndarray, ref: np.ndarray) -> np.ndarray:
@@ -150,9 +151,11 @@ def check_confidence_and_commit(cfg, step, d, inp, ref, window_len=None):
     return excluded
 
 
-def full_parity(cfg, inp, *, attn_impl="auto", window_len=None, remaining_budget=None):
-    step, d = run_gpu_step(cfg, inp, attn_impl=attn_impl, window_len=window_len, remaining_budget=remaining_budget)
-    ref = oracle_step(cfg, inp, window_len=window_len, remaining_budget=remaining_budget)
+def full_parity(cfg, inp, *, attn_impl="auto", window_len=None, remaining_budget=None, commit_mode="streaming"):
+    step, d = run_gpu_step(cfg, inp, attn_impl=attn_impl, window_len=window_len, remaining_budget=remaining_budget,
+                           commit_mode=commit_mode)
+    ref = oracle_step(cfg, inp, window_len=window_len, remaining_budget=remaining_budget,
+                      block_commit=(commit_mode == "block"))
     check_reorder(step, ref)
     err = check_attention(cfg, step, d, inp, ref)
     excluded = check_confidence_and_commit(cfg, step, d, inp, ref, window_len)

@@ -45,6 +45,27 @@ def test_tiny_model_text_is_token_exact(W, tilt, tau):
         assert got["steps"] < N
 
 
+@pytest.mark.parametrize("W,tilt,tau", [(4, 8.0, 0.5), (8, 30.0, 0.35)])
+def test_tiny_model_block_wise_baseline_is_token_exact(W, tilt, tau):
+    from paper_2512_22737_b200.loop import StreamingDecoder
+    B, P, N = 2, 21, 26
+    wts = make_model(TINY)
+    pt = make_prompts_and_targets(TINY, B, P, N)
+    dec = StreamingDecoder(TINY, wts, batch=B, window=W, max_total_len=P + N, tau=tau, lam=0.1, tilt=tilt,
+                           target=pt["target"], commit_mode="block")
+    dec.prefill(pt["prompt"])
+    # prefill windows are fully filled, so the block rule commits them whole as well
+    assert dec.prefix_len.cpu().tolist() == [P] * B
+    got = dec.generate(N)
+    n_fwd_ref = 0
+    for b in range(B):
+        ref = mo.decode(wts, TINY, pt["prompt"][b], pt["target"][b], tilt=tilt, window=W, max_new_tokens=N,
+                        conf_mode="entropy", tau=tau, lam=0.1, maxprob_thr=0.9, block_commit=True)
+        assert got["y"][b] == ref["y"]
+        n_fwd_ref += ref["n_fwd"]
+    assert got["n_fwd"] == n_fwd_ref
+
+
 def _bits(t):
     return t.view(torch.int16).cpu().numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.cpu().numpy()
 

@@ -338,3 +338,16 @@ def test_a_wait_that_nothing_satisfies_expires_and_reports_status():
     import parity_util as pu
     cfg = _small_qwen(batch=1, window=8, prefix_lo=40, prefix_hi=40, vocab=1024, name="afterwait")
     pu.full_parity(cfg, make_step(cfg, seed=2))
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_block_wise_commit_mode(impl):
+    """WEDLM_COMMIT_BLOCK: nothing is committed unless every active slot is filled."""
+    import parity_util as pu
+    cfg = _small_qwen(batch=4, window=8, prefix_lo=30, prefix_hi=200, vocab=2048, boost=14.0, boost_prob=0.8,
+                      name="blockmode")
+    f = np.array([[1, 1, 1, 1, 1, 1, 1, 1], [1, 1, 0, 1, 0, 0, 1, 1], [0, 0, 0, 0, 0, 0, 0, 0], [1, 1, 1, 1, 1, 0, 0, 0]], np.uint8)
+    inp = make_step(cfg, seed=51, filled=f)
+    r = pu.full_parity(cfg, inp, attn_impl=impl, window_len=[8, 8, 8, 5], remaining_budget=[50, 50, 50, 2],
+                       commit_mode="block")
+    assert r["step"].committed_count.cpu().tolist() == [8, 0, 0, 5]

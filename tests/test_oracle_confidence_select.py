@@ -201,3 +201,42 @@ def test_step_function_composes_the_parts():
         assert ps["committed_tokens"] == inp["window_tokens"][b][: ps["committed_count"]].tolist()
         assert ps["filled_count"] >= 1 or r["n_filled"][b] == W
         assert ps["window_len"] == W
+
+
+# ------------------------------------------------------------------ block-wise baseline
+def test_block_wise_baseline_commits_all_or_nothing():
+    """Hand-worked against the description of block decoding (Section 5.2, Fig. 2): [A,B,M,M] commits
+    nothing although A,B lead the window; once the block is complete it is committed whole."""
+    kw = dict(conf_mode="entropy", tau=0.5, lam=0.1, maxprob_thr=0.9, mask_token_id=99, block_commit=True)
+    r = orc.select_commit_refill([11, 12, 99, 99], [1, 1, 0, 0], 4, 20, [7, 8], [0.1, 0.9], [0.9, 0.5], **kw)
+    assert r["committed_count"] == 0 and r["committed_tokens"] == []
+    assert r["window_tokens"] == [11, 12, 7, 99] and r["filled"] == [1, 1, 1, 0]
+    assert r["prefix_len"] == 20 and r["window_len"] == 4
+    r = orc.select_commit_refill([11, 12, 7, 9], [1, 1, 1, 1], 4, 20, [], [], [], **kw)
+    assert r["committed_tokens"] == [11, 12, 7, 9] and r["prefix_len"] == 24
+    assert r["window_tokens"] == [99, 99, 99, 99] and r["filled"] == [0, 0, 0, 0]
+    ro = orc.reorder(np.array([[1, 1, 0, 0], [1, 1, 1, 1]], np.uint8), np.array([20, 20]), block_commit=True)
+    assert ro["n_commit"].tolist() == [0, 4]
+
+
+def test_block_wise_loop_produces_the_same_text():
+    """With logits that depend on the position only, streaming and block-wise decoding write the same
+    text; the block-wise loop commits in whole blocks only."""
+    V, P, N, W = 40, 5, 33, 8
+    rows = {}
+
+    def forward(y, toks, pos):
+        out = []
+        for p in pos:
+            if p not in rows:
+                rows[p] = np.random.default_rng(p).standard_normal(V) * (4.0 if p % 3 else 0.5)
+            out.append(rows[p])
+        return np.stack(out)
+
+    kw = dict(prefix_len=P, window=W, max_new_tokens=N, conf_mode="entropy", tau=2.0, lam=0.05, maxprob_thr=0.9,
+              mask_token_id=V - 1)
+    a = orc.decode_loop(forward, **kw)
+    b = orc.decode_loop(forward, block_commit=True, **kw)
+    assert a["y"] == b["y"] and len(a["y"]) == N
+    assert all(tr["committed"] in (0, tr["window_len"]) for tr in b["trace"])
+    assert any(0 < tr["committed"] < tr["window_len"] for tr in a["trace"])
