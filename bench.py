@@ -539,8 +539,8 @@ def run_loop(args):
     runs = [(W, "streaming") for W in args.loop_windows] + [(W, "block") for W in args.loop_block_windows]
     for W, mode in runs:
         for tilt_name, tilt in args.loop_tilts:
-            dec = StreamingDecoder(m, {}, batch=B, window=W, max_total_len=P + N, tau=0.3, lam=0.1, tilt=0.0,
-                                   target=pt["target"], commit_mode=mode)
+            dec = StreamingDecoder(m, {}, batch=B, window=W, max_total_len=P + N, tau=args.loop_tau, lam=args.loop_lambda,
+                                   tilt=0.0, target=pt["target"], commit_mode=mode)
             dec.wt = wts
             dec.prefill(pt["prompt"])
             if lse0 is None:                    # log-sum-exp of the untilted logits, measured once
@@ -563,6 +563,7 @@ def run_loop(args):
             torch.cuda.empty_cache()
     line = {"metric": "generated_tokens_per_s", "unit": "tokens/s", "n_gpus": 1, "data": "synthetic", "dtype": "bf16",
             "config": {"workload": "cfg5_loop", "batch": B, "prompt": P, "new_tokens": N, "layers": m.n_layers,
+                       "tau": args.loop_tau, "lambda": args.loop_lambda,
                        "hidden": H, "lse_of_untilted_logits": lse0,
                        "timing": "host wall clock around generate(), includes the per-step read-back of commits"},
             "results": results}
@@ -585,6 +586,8 @@ def main():
     ap.add_argument("--loop-batch", type=int, default=16)
     ap.add_argument("--loop-new-tokens", type=int, default=1024)
     ap.add_argument("--loop-windows", type=lambda s: [int(x) for x in s.split(",")], default=[16, 2, 1])
+    ap.add_argument("--loop-tau", type=float, default=0.3)
+    ap.add_argument("--loop-lambda", type=float, default=0.1)
     ap.add_argument("--loop-block-windows", type=lambda s: [int(x) for x in s.split(",") if x], default=[16],
                     help="windows also run with the block-wise commit rule (the baseline of Fig. 3c)")
     ap.add_argument("--loop-tilts", type=lambda s: [(t.split(":")[0], float(t.split(":")[1])) for t in s.split(",")],
