@@ -61,8 +61,10 @@ struct TensorAttnParams {
 };
 
 #ifdef WEDLM_ATTN_TRACE
+}  // namespace
 // Debug builds only: per-tile timestamps of one CTA, [role][tile][event].
 __device__ long long g_attn_trace[4 * 256 * 8];
+namespace {
 #define TRACE(role, t, ev) do { if (trace_on && (unsigned)(t) < 256u) g_attn_trace[((role) * 256 + (t)) * 8 + (ev)] = clock64(); } while (0)
 #else
 #define TRACE(role, t, ev) do { } while (0)
@@ -428,6 +430,7 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         m_tile = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
       }
+      TRACE(2, t, 7);
       // lazy reference: only move it when the maximum grew by more than 2^kLazyRescaleLog2
       float alpha = 1.f;
       bool moved = false;
@@ -600,15 +603,13 @@ int launch_wait_expiry_selftest(uint32_t max_polls, int32_t* status, cudaStream_
   return cuda_ok(cudaGetLastError());
 }
 
-namespace {
-
 #ifdef WEDLM_ATTN_TRACE
+}  // namespace wedlm
 extern "C" int wedlm_debug_read_attn_trace(long long* host_dst) {
-  return cudaMemcpyFromSymbol(host_dst, g_attn_trace, sizeof(long long) * 4 * 256 * 8) == cudaSuccess ? 0 : -4;
+  return cudaMemcpyFromSymbol(host_dst, wedlm::g_attn_trace, sizeof(long long) * 4 * 256 * 8) == cudaSuccess ? 0 : -4;
 }
+namespace wedlm {
 #endif
-
-}  // namespace
 
 bool attn_tensor_supported(const wedlm_config_t* c) {
   if (c->dtype != WEDLM_DTYPE_BF16 || c->head_dim != kD || c->page_size != kPage) return false;
