@@ -536,12 +536,15 @@ def run_loop(args):
     pt = make_prompts_and_targets(m, B, P, N)
     results = []
     lse0 = None
-    runs = [(W, "streaming") for W in args.loop_windows] + [(W, "block") for W in args.loop_block_windows]
-    for W, mode in runs:
+    runs = [(W, "streaming", False) for W in args.loop_windows] + [(W, "block", False) for W in args.loop_block_windows] + \
+           [(W, "streaming", True) for W in args.loop_fused_windows]
+    lm_head_vh = wts["lm_head"].t().contiguous() if args.loop_fused_windows else None
+    for W, mode, fused in runs:
         for tilt_name, tilt in args.loop_tilts:
             dec = StreamingDecoder(m, {}, batch=B, window=W, max_total_len=P + N, tau=args.loop_tau, lam=args.loop_lambda,
-                                   tilt=0.0, target=pt["target"], commit_mode=mode)
+                                   tilt=0.0, target=pt["target"], commit_mode=mode, fused_lm_head=fused)
             dec.wt = wts
+            dec.lm_head_vh = lm_head_vh
             dec.prefill(pt["prompt"])
             if lse0 is None:                    # log-sum-exp of the untilted logits, measured once
                 dec.start(N)
@@ -555,7 +558,8 @@ def run_loop(args):
             dt = time.perf_counter() - t0
             n_gen = sum(len(y) for y in out["y"])
             on_target = sum(int(out["y"][bb] == pt["target"][bb, P:P + N].tolist()) for bb in range(B))
-            results.append({"window": W, "commit": mode, "tilt": f"{tilt_name}+{tilt:g}", "tokens_per_s": n_gen / dt, "seconds": dt,
+            results.append({"window": W, "commit": mode, "lm_head": "fused" if fused else "gemm+logits",
+                            "tilt": f"{tilt_name}+{tilt:g}", "tokens_per_s": n_gen / dt, "seconds": dt,
                             "steps": out["steps"], "tokens_per_step_per_seq": n_gen / B / max(out["steps"], 1),
                             "p_cache": out["p_cache"], "sequences_equal_to_target": on_target})
             log(results[-1])
@@ -586,6 +590,8 @@ def main():
     ap.add_argument("--loop-batch", type=int, default=16)
     ap.add_argument("--loop-new-tokens", type=int, default=1024)
     ap.add_argument("--loop-windows", type=lambda s: [int(x) for x in s.split(",")], default=[16, 2, 1])
+    ap.add_argument("--loop-fused-windows", type=lambda s: [int(x) for x in s.split(",") if x], default=[],
+                    help="windows also run with the LM head fused into the confidence call")
     ap.add_argument("--loop-tau", type=float, default=0.3)
     ap.add_argument("--loop-lambda", type=float, default=0.1)
     ap.add_argument("--loop-block-windows", type=lambda s: [int(x) for x in s.split(",") if x], default=[16],

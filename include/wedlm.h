@@ -211,6 +211,29 @@ int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const
                             void* stream);
 
 /*
+ * wedlm_confidence_commit fused with the LM head (Algorithm 1 takes its logits from Forward; here the last
+ * step of that forward, logits = hidden . lm_head^T, is computed tile by tile on the tensor cores and reduced
+ * in place, so the [B,W,V] logits never exist in memory).  bf16 only; hidden must be a multiple of 64.
+ *   hidden        H
+ *   hidden_states in  bf16 [B,W,H]  physical order (after the model's final norm)
+ *   lm_head       in  bf16 [V,H]    row v = output embedding of token v
+ *   tilt_ids      in  i32  [B,W] or NULL: the logit of token tilt_ids[b,i] of physical row i gets +tilt
+ *                 (the additive tilt toward a target sequence of the end-to-end configuration); -1 = none
+ *   all other arguments as in wedlm_confidence_commit; statistics come from fp32 logits (not rounded to bf16).
+ * Workspace: wedlm_lmhead_confidence_workspace_bytes(cfg) = batch*window*ceil(vocab/128)*16 bytes.
+ */
+size_t wedlm_lmhead_confidence_workspace_bytes(const wedlm_config_t* cfg);
+int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, const void* hidden_states,
+                                   const void* lm_head, const int32_t* tilt_ids, float tilt,
+                                   const int32_t* perm, const int32_t* n_filled, const int32_t* n_commit,
+                                   int32_t* window_tokens, uint8_t* filled, int32_t* prefix_len,
+                                   int32_t* window_len, int32_t* remaining_budget,
+                                   int32_t* argmax, float* maxprob, float* entropy, float* lse,
+                                   int32_t* committed_tokens, int32_t* committed_count,
+                                   int32_t* filled_count, void* workspace, size_t workspace_bytes,
+                                   void* stream);
+
+/*
  * wedlm_confidence_commit without a workspace argument, for hosts that must not allocate device
  * memory while they run.  (The paper has no counterpart to this call; it exists for deployment.)
  *

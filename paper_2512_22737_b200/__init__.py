@@ -19,6 +19,8 @@ from .binding import (  # noqa: F401
     wedlm_confidence_workspace_bytes,
     wedlm_kv_append,
     wedlm_launch_count,
+    wedlm_lmhead_confidence_commit,
+    wedlm_lmhead_confidence_workspace_bytes,
     wedlm_profile_next_attn,
     wedlm_reorder,
     wedlm_selftest_wait_expiry,

@@ -92,6 +92,12 @@ def load_library() -> ctypes.CDLL:
     lib.wedlm_confidence_commit_static.restype = ctypes.c_int
     lib.wedlm_confidence_commit_static.argtypes = [cfgp, vp, i32p, i32p, i32p, i32p, u8p, i32p, i32p, i32p,
                                                    i32p, f32p, f32p, f32p, i32p, i32p, i32p, vp]
+    lib.wedlm_lmhead_confidence_workspace_bytes.restype = ctypes.c_size_t
+    lib.wedlm_lmhead_confidence_workspace_bytes.argtypes = [cfgp]
+    lib.wedlm_lmhead_confidence_commit.restype = ctypes.c_int
+    lib.wedlm_lmhead_confidence_commit.argtypes = [cfgp, ctypes.c_int32, vp, vp, i32p, ctypes.c_float, i32p, i32p, i32p,
+                                                   i32p, u8p, i32p, i32p, i32p, i32p, f32p, f32p, f32p, i32p, i32p,
+                                                   i32p, vp, ctypes.c_size_t, vp]
     lib.wedlm_window_refill.restype = ctypes.c_int
     lib.wedlm_window_refill.argtypes = [cfgp, i32p, i32p, u8p, i32p, i32p, i32p, i32p, i32p, vp]
     _lib = lib
@@ -225,6 +231,27 @@ def wedlm_confidence_commit(cfg, logits, perm, n_filled, n_commit, window_tokens
         _ptr(committed_count, i32, "committed_count"), _ptr(filled_count, i32, "filled_count"),
         _ptr(workspace, None, "workspace"), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
         _stream(stream)), "wedlm_confidence_commit")
+
+
+def wedlm_lmhead_confidence_workspace_bytes(cfg) -> int:
+    return int(load_library().wedlm_lmhead_confidence_workspace_bytes(ctypes.byref(cfg)))
+
+
+def wedlm_lmhead_confidence_commit(cfg, hidden_states, lm_head, tilt_ids, tilt, perm, n_filled, n_commit, window_tokens,
+                                   filled, prefix_len, window_len, remaining_budget, argmax, maxprob, entropy, lse,
+                                   committed_tokens, committed_count, filled_count, workspace, stream=None) -> None:
+    """Confidence/commit straight from the hidden states [B,W,H] and the output embedding [V,H] (bf16)."""
+    i32, u8, f32, bf = torch.int32, torch.uint8, torch.float32, torch.bfloat16
+    _check(load_library().wedlm_lmhead_confidence_commit(
+        ctypes.byref(cfg), ctypes.c_int32(hidden_states.shape[-1]), _ptr(hidden_states, bf, "hidden_states"),
+        _ptr(lm_head, bf, "lm_head"), _ptr(tilt_ids, i32, "tilt_ids"), ctypes.c_float(tilt), _ptr(perm, i32, "perm"),
+        _ptr(n_filled, i32, "n_filled"), _ptr(n_commit, i32, "n_commit"), _ptr(window_tokens, i32, "window_tokens"),
+        _ptr(filled, u8, "filled"), _ptr(prefix_len, i32, "prefix_len"), _ptr(window_len, i32, "window_len"),
+        _ptr(remaining_budget, i32, "remaining_budget"), _ptr(argmax, i32, "argmax"), _ptr(maxprob, f32, "maxprob"),
+        _ptr(entropy, f32, "entropy"), _ptr(lse, f32, "lse"), _ptr(committed_tokens, i32, "committed_tokens"),
+        _ptr(committed_count, i32, "committed_count"), _ptr(filled_count, i32, "filled_count"),
+        _ptr(workspace, None, "workspace"), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+        _stream(stream)), "wedlm_lmhead_confidence_commit")
 
 
 WEDLM_STATIC_SCRATCH_BYTES = 4 << 20

@@ -244,6 +244,37 @@ int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const
                            committed_count, filled_count, workspace, (cudaStream_t)stream);
 }
 
+size_t wedlm_lmhead_confidence_workspace_bytes(const wedlm_config_t* cfg) {
+  if (check_config(cfg, false, true) != WEDLM_OK) return 0;
+  size_t b = (size_t)cfg->batch * cfg->window * lmhead_conf_tiles(cfg->vocab) * 16;
+  return b ? b : 256;
+}
+
+int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, const void* hidden_states,
+                                   const void* lm_head, const int32_t* tilt_ids, float tilt, const int32_t* perm,
+                                   const int32_t* n_filled, const int32_t* n_commit, int32_t* window_tokens,
+                                   uint8_t* filled, int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
+                                   int32_t* argmax, float* maxprob, float* entropy, float* lse, int32_t* committed_tokens,
+                                   int32_t* committed_count, int32_t* filled_count, void* workspace, size_t workspace_bytes,
+                                   void* stream) {
+  int rc = check_config(cfg, false, true);
+  if (rc != WEDLM_OK) return rc;
+  if (cfg->dtype != WEDLM_DTYPE_BF16 || hidden < 64 || hidden % 64 != 0) return WEDLM_ERR_UNSUPPORTED;
+  if ((long long)cfg->batch * cfg->window >= (1ll << 31) / 2) return WEDLM_ERR_UNSUPPORTED;
+  if (cfg->batch == 0) return WEDLM_OK;
+  if (!hidden_states || !lm_head || !perm || !n_filled || !n_commit || !window_tokens || !filled || !prefix_len || !workspace)
+    return WEDLM_ERR_INVALID_ARG;
+  if (!aligned16(hidden_states) || !aligned16(lm_head) || !aligned16(workspace)) return WEDLM_ERR_INVALID_ARG;
+  if (workspace_bytes < wedlm_lmhead_confidence_workspace_bytes(cfg)) return WEDLM_ERR_WORKSPACE_TOO_SMALL;
+  Shape s = make_shape(cfg);
+  cudaStream_t st = (cudaStream_t)stream;
+  rc = launch_lmhead_conf(s, hidden, hidden_states, lm_head, tilt_ids, tilt, n_filled, window_len, workspace, st);
+  if (rc != WEDLM_OK) return rc;
+  return launch_conf_commit(s, cfg, lmhead_conf_tiles(cfg->vocab), workspace, perm, n_filled, n_commit, window_tokens, filled,
+                            prefix_len, window_len, remaining_budget, argmax, maxprob, entropy, lse, committed_tokens,
+                            committed_count, filled_count, st);
+}
+
 int wedlm_window_refill(const wedlm_config_t* cfg, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
                         int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
                         int32_t* committed_tokens, int32_t* committed_count, void* stream) {

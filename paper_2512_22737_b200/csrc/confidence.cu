@@ -604,13 +604,25 @@ int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* log
   }
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return WEDLM_ERR_CUDA;
+  return launch_conf_commit(s, cfg, n_chunks, part, perm, n_filled, n_commit, window_tokens, filled, prefix_len, window_len,
+                            remaining_budget, argmax, maxprob, entropy, lse, committed_tokens, committed_count,
+                            filled_count, st);
+}
+
+// Pass 2 alone: merge `n_chunks` partials (m, s, t, argmax) per mask row, select, commit, refill.
+int launch_conf_commit(const Shape& s, const wedlm_config_t* cfg, int n_chunks, const void* partials, const int32_t* perm,
+                       const int32_t* n_filled, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
+                       int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget, int32_t* argmax,
+                       float* maxprob, float* entropy, float* lse, int32_t* committed_tokens, int32_t* committed_count,
+                       int32_t* filled_count, cudaStream_t st) {
   ConfParams p{s.W, n_chunks, cfg->conf_mode, cfg->mask_token_id, cfg->tau, cfg->lambda, cfg->maxprob_thr};
   size_t smem = (size_t)s.W * (sizeof(double) + 2 * sizeof(int) + 2);
   int commit_threads = 32 * s.W;
   commit_threads = commit_threads < 128 ? 128 : (commit_threads > 1024 ? 1024 : commit_threads);
-  conf_commit_kernel<<<s.B, commit_threads, smem, st>>>(p, part, perm, n_filled, n_commit, window_tokens, filled, prefix_len,
-                                            window_len, remaining_budget, argmax, maxprob, entropy, lse,
-                                            committed_tokens, committed_count, filled_count);
+  conf_commit_kernel<<<s.B, commit_threads, smem, st>>>(p, reinterpret_cast<const float4*>(partials), perm, n_filled, n_commit,
+                                                        window_tokens, filled, prefix_len, window_len, remaining_budget,
+                                                        argmax, maxprob, entropy, lse, committed_tokens, committed_count,
+                                                        filled_count);
   count_launch();
   return cuda_ok(cudaGetLastError());
 }

@@ -27,7 +27,8 @@ class StreamingDecoder:
     def __init__(self, mcfg, weights: Dict[str, np.ndarray], *, batch: int, window: int, max_total_len: int,
                  conf_mode: str = "entropy", tau: float = 0.3, lam: float = 0.1, maxprob_thr: float = 0.9,
                  tilt: float = 0.0, target: Optional[np.ndarray] = None, page_size: int = 16,
-                 attn_impl: str = "auto", seed: int = 0, commit_mode: str = "streaming"):
+                 attn_impl: str = "auto", seed: int = 0, commit_mode: str = "streaming",
+                 fused_lm_head: bool = False):
         self.m = mcfg
         self.B, self.W = batch, window
         self.dtype = torch.bfloat16 if mcfg.dtype == "bf16" else torch.float32
@@ -50,6 +51,14 @@ class StreamingDecoder:
             maxprob_thr=maxprob_thr, mask_token_id=mcfg.mask_token_id, max_prefix_len=max_total_len,
             attn_impl=attn_impl, commit_mode=commit_mode)
         self.step_bufs = w.DecodeStep(self.cfg)
+        # fused LM head: logits are never materialised; the output embedding is kept as [V, H]
+        self.fused_lm_head = fused_lm_head
+        self.lm_head_vh = None
+        self.lm_ws = None
+        if fused_lm_head:
+            if "lm_head" in self.wt:
+                self.lm_head_vh = self.wt["lm_head"].t().contiguous()
+            self.lm_ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(self.cfg), dtype=torch.uint8, device="cuda")
         i32 = dict(dtype=torch.int32, device="cuda")
         self.window_tokens = torch.full((batch, window), mcfg.mask_token_id, **i32)
         self.filled = torch.zeros(batch, window, dtype=torch.uint8, device="cuda")
@@ -65,8 +74,9 @@ class StreamingDecoder:
         y = xf * torch.rsqrt(xf.pow(2).mean(-1, keepdim=True) + self.m.rms_eps)
         return (y * gain.float()).to(self.dtype)
 
-    def forward(self, capture_layer: Optional[int] = None):
-        """Causal forward of the reordered window on top of the cache -> logits [B, W, V]."""
+    def forward(self, capture_layer: Optional[int] = None, want_logits: bool = True):
+        """Causal forward of the reordered window on top of the cache -> logits [B, W, V] (or, with
+        want_logits=False, the normalised hidden states [B, W, H] that feed the LM head)."""
         s, m = self.step_bufs, self.m
         B, W = self.B, self.W
         s.reorder(self.filled, self.window_tokens, self.prefix_len, self.window_len)
@@ -87,7 +97,10 @@ class StreamingDecoder:
             h = h + s.out.view(B, W, -1) @ self.wt[f"l{l}.wo"]
             mm = self._rms(h, self.wt[f"l{l}.norm2"])
             h = h + (torch.nn.functional.silu(mm @ self.wt[f"l{l}.wg"]) * (mm @ self.wt[f"l{l}.wu"])) @ self.wt[f"l{l}.wd"]
-        logits = self._rms(h, self.wt["norm_f"]) @ self.wt["lm_head"]
+        hn = self._rms(h, self.wt["norm_f"])
+        if not want_logits:
+            return hn.contiguous(), cap
+        logits = hn @ self.wt["lm_head"]
         if self.tilt != 0.0 and self.target is not None:
             pos = s.pos_ids.long().clamp_(max=self.target.shape[1] - 1)
             idx = self.target.gather(1, pos)                                 # [B, W] target id at each row's position
@@ -133,6 +146,20 @@ class StreamingDecoder:
             snap = dict(filled=self.filled.clone(), window_tokens=self.window_tokens.clone(),
                         prefix_len=self.prefix_len.clone(), window_len=self.window_len.clone(),
                         budget=self.budget.clone())
+        if self.fused_lm_head and capture_layer is None:
+            hn, cap = self.forward(None, want_logits=False)
+            tilt_ids = None
+            if self.tilt != 0.0 and self.target is not None:
+                pos = s.pos_ids.long().clamp_(max=self.target.shape[1] - 1)
+                tilt_ids = self.target.gather(1, pos).to(torch.int32)
+            if self.lm_head_vh is None:
+                self.lm_head_vh = self.wt["lm_head"].t().contiguous()
+            w.wedlm_lmhead_confidence_commit(self.cfg, hn, self.lm_head_vh, tilt_ids, float(self.tilt), s.perm, s.n_filled,
+                                             s.n_commit, self.window_tokens, self.filled, self.prefix_len, self.window_len,
+                                             self.budget, s.argmax, s.maxprob, s.entropy, s.lse, s.committed_tokens,
+                                             s.committed_count, s.filled_count, self.lm_ws)
+            self.steps += 1
+            return s.committed_count, s.committed_tokens
         logits, cap = self.forward(capture_layer)
         s.confidence_commit(logits, self.window_tokens, self.filled, self.prefix_len, self.window_len, self.budget)
         self.steps += 1

@@ -1,0 +1,87 @@
+"""The fused LM head + confidence/commit call against the oracle: logits = hidden . lm_head^T in float64
+from the same bf16 bit patterns, then the oracle's confidence / selection / commit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import wedlm_oracle as orc
+from workloads import StepConfig, bf16_bits, make_step
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(B, W, V, H, seed, boost=6.0, window_len=None, budget=None, commit_mode="streaming"):
+    import paper_2512_22737_b200 as w
+    import parity_util as pu
+    cfg = StepConfig(name="lmhead", batch=B, window=W, n_q_heads=4, n_kv_heads=1, head_dim=128, vocab=V, dtype="bf16",
+                     prefix_lo=10, prefix_hi=60, obs_prob_lo=0.2, obs_prob_hi=0.6, tau=0.3, lam=0.1)
+    inp = make_step(cfg, seed=seed, with_logits=False)
+    g = np.random.default_rng(seed)
+    hid = bf16_bits((g.standard_normal((B, W, H)) * 1.0).astype(np.float32).reshape(-1)).reshape(B, W, H)
+    emb = bf16_bits((g.standard_normal((V, H)) * (2.0 / np.sqrt(H))).astype(np.float32).reshape(-1)).reshape(V, H)
+    tilt_ids = g.integers(0, V - 1, size=(B, W)).astype(np.int32)
+    tilt_ids[g.random((B, W)) < 0.3] = -1
+    # oracle logits in float64 from the bf16 inputs, tilt added where asked
+    logits = orc.to_f64(hid) @ orc.to_f64(emb).T
+    bb, ww = np.nonzero(tilt_ids >= 0)
+    logits[bb, ww, tilt_ids[bb, ww]] += boost
+    inp["logits"] = logits
+    ref = pu.oracle_step(cfg, inp, window_len=window_len, remaining_budget=budget, with_attention=False,
+                         block_commit=(commit_mode == "block"))
+    # GPU
+    c = w.config_for(cfg, max_pages_per_seq=inp["block_table"].shape[1], num_pages=inp["k_cache"].shape[0],
+                     max_prefix_len=int(inp["prefix_len"].max()), commit_mode=commit_mode)
+    step = w.DecodeStep(c)
+    d = {k: w.to_device(inp[k]) for k in ("filled", "window_tokens", "prefix_len")}
+    wl = None if window_len is None else torch.tensor(window_len, dtype=torch.int32, device="cuda")
+    bud = None if budget is None else torch.tensor(budget, dtype=torch.int32, device="cuda")
+    step.reorder(d["filled"], d["window_tokens"], d["prefix_len"], wl)
+    ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c), dtype=torch.uint8, device="cuda")
+    w.wedlm_lmhead_confidence_commit(c, w.to_device(hid), w.to_device(emb), w.to_device(tilt_ids), boost, step.perm,
+                                     step.n_filled, step.n_commit, d["window_tokens"], d["filled"], d["prefix_len"], wl, bud,
+                                     step.argmax, step.maxprob, step.entropy, step.lse, step.committed_tokens,
+                                     step.committed_count, step.filled_count, ws)
+    torch.cuda.synchronize()
+    d["window_len"], d["remaining_budget"] = wl, bud
+    # arg-max: exact unless the two best logits of the row are within the 1e-3 band
+    am = step.argmax.cpu().numpy()
+    near_tie = 0
+    for b in range(B):
+        for i in range(W):
+            if ref["argmax"][b, i] >= 0 and am[b, i] != ref["argmax"][b, i]:
+                top2 = np.sort(logits[b, i])[-2:]
+                assert top2[1] - top2[0] <= 1e-3, (b, i, am[b, i], ref["argmax"][b, i], top2)
+                near_tie += 1
+                ref["argmax"][b, i] = am[b, i]
+    assert near_tie == 0 or near_tie <= 2
+    if near_tie == 0:
+        pu.check_confidence_and_commit(cfg, step, d, inp, ref, window_len)
+    return step, ref
+
+
+@pytest.mark.parametrize("B,W,V,H", [(2, 8, 1000, 64), (3, 16, 5000, 256), (1, 40, 4096, 512), (5, 64, 3333, 128)])
+def test_fused_lmhead_confidence_matches_oracle(B, W, V, H):
+    _case(B, W, V, H, seed=B * 100 + W)
+
+
+def test_fused_lmhead_short_windows_budget_and_block_mode():
+    _case(4, 8, 2048, 128, seed=9, window_len=[8, 5, 3, 8], budget=[10, 1, 0, 10])
+    _case(4, 8, 2048, 128, seed=10, commit_mode="block")
+
+
+def test_fused_lmhead_qwen_width_rows_over_256():
+    """Hidden 4096 (64 k-steps through the 4-stage ring) and more than 256 rows (two row chunks)."""
+    _case(10, 32, 8192, 4096, seed=11, boost=14.0)
+
+
+def test_fused_lmhead_rejects_unsupported_shapes():
+    import paper_2512_22737_b200 as w
+    c = w.make_config(batch=1, window=8, vocab=1000, dtype="bf16")
+    x = torch.zeros(8 * 96, dtype=torch.bfloat16, device="cuda").view(1, 8, 96)        # hidden not a multiple of 64
+    e = torch.zeros(8, dtype=torch.int32, device="cuda")
+    ws = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(w.WedlmError) as err:
+        w.wedlm_lmhead_confidence_commit(c, x, torch.zeros(1000, 96, dtype=torch.bfloat16, device="cuda"), None, 0.0, e, e, e,
+                                         e, torch.zeros(8, dtype=torch.uint8, device="cuda"), e, None, None, None, None, None,
+                                         None, None, None, None, ws)
+    assert err.value.code == -2

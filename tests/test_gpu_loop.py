@@ -120,3 +120,24 @@ def test_bf16_loop_replays_every_step_against_the_oracle(impl):
         assert ys[b] == pt["target"][b, P:P + N].tolist()          # tilt 14 dominates a random-init model
     assert steps < N                                                  # several tokens per step
     print(f"{impl}: {steps} steps for {N} tokens, worst attention error {worst:.2e}, excluded decisions {excluded}")
+
+
+def test_fused_lm_head_loop_writes_the_same_text():
+    """The loop with the LM head fused into the confidence call (no logits tensor) against the loop that
+    materialises bf16 logits: same committed text when the tilt decides the tokens, same number of tokens."""
+    from paper_2512_22737_b200.loop import StreamingDecoder
+    m = ModelConfig(name="small_bf16", vocab=4096, hidden=256, n_layers=2, n_q_heads=8, n_kv_heads=2, head_dim=128,
+                    ffn=512, dtype="bf16", rope_theta=1.0e6, init_std=0.05)
+    B, W, P, N = 3, 16, 40, 40
+    wts = make_model(m, seed=7)
+    pt = make_prompts_and_targets(m, B, P, N, seed=7)
+    outs = []
+    for fused in (False, True):
+        dec = StreamingDecoder(m, wts, batch=B, window=W, max_total_len=P + N, tau=0.35, lam=0.1, tilt=16.0,
+                               target=pt["target"], fused_lm_head=fused)
+        dec.prefill(pt["prompt"])
+        outs.append(dec.generate(N))
+    for b in range(B):
+        assert outs[1]["y"][b] == pt["target"][b, P:P + N].tolist()
+        assert outs[0]["y"][b] == outs[1]["y"][b]
+    assert outs[1]["steps"] < N
