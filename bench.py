@@ -575,6 +575,59 @@ def run_loop(args):
     return 0
 
 
+def run_lmhead(args):
+    """LM head + confidence/commit at the end-to-end configuration's shape (16 x 16 rows, hidden 4096, vocabulary
+    151 936): the fused call (logits stay in tensor memory) against a library GEMM that writes bf16 logits
+    followed by the streaming confidence call."""
+    import torch
+    from paper_2512_22737_b200 import build as b
+    b.build()
+    import paper_2512_22737_b200 as w
+    torch.cuda.set_device(0)
+    B, W, V, H = 16, 16, 151936, 4096
+    torch.manual_seed(0)
+    hid = torch.randn(B, W, H, device="cuda").to(torch.bfloat16)
+    emb = (torch.randn(V, H, device="cuda") * 0.02).to(torch.bfloat16)
+    emb_hv = emb.t().contiguous()
+    c = w.make_config(batch=B, window=W, n_q_heads=32, n_kv_heads=8, head_dim=128, max_pages_per_seq=4, num_pages=64,
+                      vocab=V, dtype="bf16", mask_token_id=V - 1, max_prefix_len=16)
+    step = w.DecodeStep(c)
+    filled = (torch.rand(B, W, device="cuda") < 0.3).to(torch.uint8)
+    tok = torch.zeros(B, W, dtype=torch.int32, device="cuda")
+    pl = torch.full((B,), 16, dtype=torch.int32, device="cuda")
+    step.reorder(filled, tok, pl)
+    ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c), dtype=torch.uint8, device="cuda")
+
+    def fused(f, t, p):
+        w.wedlm_lmhead_confidence_commit(c, hid, emb, None, 0.0, step.perm, step.n_filled, step.n_commit, t, f, p, None, None,
+                                         step.argmax, step.maxprob, step.entropy, step.lse, step.committed_tokens,
+                                         step.committed_count, step.filled_count, ws)
+
+    def unfused(f, t, p):
+        step.confidence_commit((hid @ emb_hv).contiguous(), t, f, p)
+
+    out = {}
+    for name, fn in (("fused", fused), ("gemm_then_confidence", unfused)):
+        ts = []
+        for _ in range(args.warmup + args.steps):
+            f, t, p = filled.clone(), tok.clone(), pl.clone()
+            a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn(f, t, p)
+            e.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(e))
+        ts = ts[args.warmup:]
+        out[name] = {"ms_min": min(ts), "ms_median": statistics.median(ts)}
+    weights = V * H * 2
+    line = {"metric": "lm_head_confidence_ms", "unit": "ms", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "lmhead", "rows": B * W, "hidden": H, "vocab": V},
+            "results": out, "weight_bytes": weights, "flops": 2 * B * W * H * V,
+            "fused_weight_stream_GBps": weights / (out["fused"]["ms_median"] * 1e-3) / 1e9}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -601,6 +654,8 @@ def main():
     args = ap.parse_args()
     if args.workload == "cfg5_loop":
         return run_loop(args)
+    if args.workload == "lmhead":
+        return run_lmhead(args)
     args.warmup = max(args.warmup, 3) if args.impl == "product" else args.warmup
     if args.impl == "reference":
         return run_reference(args)

@@ -220,7 +220,8 @@ int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const
  *   tilt_ids      in  i32  [B,W] or NULL: the logit of token tilt_ids[b,i] of physical row i gets +tilt
  *                 (the additive tilt toward a target sequence of the end-to-end configuration); -1 = none
  *   all other arguments as in wedlm_confidence_commit; statistics come from fp32 logits (not rounded to bf16).
- * Workspace: wedlm_lmhead_confidence_workspace_bytes(cfg) = batch*window*ceil(vocab/128)*16 bytes.
+ * Workspace: wedlm_lmhead_confidence_workspace_bytes(cfg) = batch*window*ceil(vocab/128)*16 bytes (an upper
+ * bound: the vocabulary tile width, 128..256, is chosen per launch).
  */
 size_t wedlm_lmhead_confidence_workspace_bytes(const wedlm_config_t* cfg);
 int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, const void* hidden_states,

@@ -268,9 +268,10 @@ int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, co
   if (workspace_bytes < wedlm_lmhead_confidence_workspace_bytes(cfg)) return WEDLM_ERR_WORKSPACE_TOO_SMALL;
   Shape s = make_shape(cfg);
   cudaStream_t st = (cudaStream_t)stream;
-  rc = launch_lmhead_conf(s, hidden, hidden_states, lm_head, tilt_ids, tilt, n_filled, window_len, workspace, st);
+  int n_tiles = 0;
+  rc = launch_lmhead_conf(s, hidden, hidden_states, lm_head, tilt_ids, tilt, n_filled, window_len, workspace, &n_tiles, st);
   if (rc != WEDLM_OK) return rc;
-  return launch_conf_commit(s, cfg, lmhead_conf_tiles(cfg->vocab), workspace, perm, n_filled, n_commit, window_tokens, filled,
+  return launch_conf_commit(s, cfg, n_tiles, workspace, perm, n_filled, n_commit, window_tokens, filled,
                             prefix_len, window_len, remaining_budget, argmax, maxprob, entropy, lse, committed_tokens,
                             committed_count, filled_count, st);
 }

@@ -90,10 +90,11 @@ int launch_conf_commit(const Shape& s, const wedlm_config_t* cfg, int n_chunks, 
                        float* maxprob, float* entropy, float* lse, int32_t* committed_tokens, int32_t* committed_count,
                        int32_t* filled_count, cudaStream_t st);
 
-// Fused LM head + confidence pass 1: partials [B*W][ceil(V/128)] from hidden states and the output embedding.
+// Fused LM head + confidence pass 1: partials [B*W][n_tiles] (n_tiles <= ceil(V/128), returned) from hidden states and the output embedding.
 int lmhead_conf_tiles(int vocab);
 int launch_lmhead_conf(const Shape& s, int hidden, const void* hidden_states, const void* lm_head, const int32_t* tilt_ids,
-                       float tilt, const int32_t* n_filled, const int32_t* window_len, void* partials, cudaStream_t st);
+                       float tilt, const int32_t* n_filled, const int32_t* window_len, void* partials, int* n_tiles_out,
+                       cudaStream_t st);
 
 int launch_window_refill(const Shape& s, const wedlm_config_t* cfg, const int32_t* n_commit, int32_t* window_tokens,
                          uint8_t* filled, int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
