@@ -14,6 +14,10 @@ What follows the paper, by function:
   window_attention         "a causal forward over the current window conditioned on the cached
                            prefix" (Section 5.2): plain softmax attention, written out.
   confidence               entropy H_i of the predicted distribution (Section 5.2), plus max-prob.
+  sample_token             Sample(l_i) of Algorithm 1 at a temperature (Section 6.1 evaluates at
+                           0.1): one draw from softmax(l / T), realised as arg-max of l / T plus
+                           Gumbel noise from a counter-based generator keyed by (seed, sequence,
+                           position, token).
   select_commit_refill     Algorithm 1, Commit / Predict / Refill, with Eq. 11 as selection score.
   step, decode_loop        the steps above in the order of Algorithm 1.
 
@@ -23,7 +27,9 @@ Readings of points the paper leaves open (all switchable by arguments):
   * selection is non-strict (H~ <= tau, p_max >= thr);
   * if no mask passes, exactly one mask is filled: the one with the best score, leftmost on ties;
   * d_i is the logical slot distance to the leftmost mask after the commit;
-  * entropy uses natural log on raw logits; Sample() is greedy arg-max, lowest index on ties;
+  * entropy uses natural log on raw logits (also when sampling: the temperature shapes the
+    draw, not the confidence); Sample() is greedy arg-max, lowest index on ties, unless a
+    temperature > 0 is given;
   * RoPE pairs (d, d + D/2) ("rotate-half"); style 1 pairs (2d, 2d+1);
   * GQA: query head h reads KV head h // (Hq // Hkv);
   * positions are 0-based: slot j of a window on a prefix of length P has position id P + j.
@@ -245,6 +251,62 @@ def confidence(logits_rows: np.ndarray) -> Dict[str, np.ndarray]:
 
 
 # ----------------------------------------------------------------------------------------
+# Sample(l_i) of Algorithm 1 at temperature T
+# ----------------------------------------------------------------------------------------
+# A draw from softmax(l / T) is the arg-max over v of l_v / T + g_v with g_v independent standard
+# Gumbel variables (the Gumbel-max identity), g = -ln(-ln u), u uniform on (0, 1).  The uniforms
+# come from a stateless generator so that a row's draw depends only on (seed, sequence index,
+# logical position, token id) and not on how the work is cut up: u = (h >> 8 + 1/2) / 2^24 with h
+# a 32-bit integer hash.  The hash is a xor-shift / odd-multiply finaliser; any implementation has
+# to reproduce these integer steps exactly to draw the same tokens.
+_M1 = np.uint32(0x7FEB352D)
+_M2 = np.uint32(0x846CA68B)
+_GOLD = np.uint32(0x9E3779B9)
+_POSMUL = np.uint32(0x85EBCA6B)
+
+
+def mix32(x) -> np.ndarray:
+    """Bijective 32-bit finaliser: x ^= x>>16; x *= M1; x ^= x>>15; x *= M2; x ^= x>>16 (mod 2^32)."""
+    x = np.asarray(x, dtype=np.uint32).copy()
+    with np.errstate(over="ignore"):
+        x ^= x >> np.uint32(16)
+        x *= _M1
+        x ^= x >> np.uint32(15)
+        x *= _M2
+        x ^= x >> np.uint32(16)
+    return x
+
+
+def sample_key(seed_lo: int, seed_hi: int, b: int, pos: int) -> np.uint32:
+    """Row key: k1 = mix32(seed_lo + GOLD * b); key = mix32(k1 ^ seed_hi ^ (POSMUL * pos))."""
+    with np.errstate(over="ignore"):
+        k1 = mix32(np.uint32(seed_lo & 0xFFFFFFFF) + _GOLD * np.uint32(b & 0xFFFFFFFF))
+        return mix32(k1 ^ np.uint32(seed_hi & 0xFFFFFFFF) ^ (_POSMUL * np.uint32(pos & 0xFFFFFFFF)))[()]
+
+
+def sample_uniforms(key, V: int) -> np.ndarray:
+    """u_v in (0, 1) for token ids 0..V-1: 24 high bits of mix32(key ^ GOLD * v), centred."""
+    with np.errstate(over="ignore"):
+        h = mix32(np.uint32(key) ^ (_GOLD * np.arange(V, dtype=np.uint32)))
+    return ((h >> np.uint32(8)).astype(np.float64) + 0.5) * 2.0 ** -24
+
+
+def sample_token(logits_row: np.ndarray, temperature: float, seed: Tuple[int, int], b: int, pos: int) -> Tuple[int, float]:
+    """(token, margin): token = arg-max_v of l_v / T + g_v (lowest v on ties); margin = best minus
+    second-best perturbed score (how far the draw is from flipping under rounding)."""
+    x = to_f64(np.asarray(logits_row)).reshape(-1)
+    u = sample_uniforms(sample_key(seed[0], seed[1], b, pos), x.shape[0])
+    z = x / float(temperature) - np.log(-np.log(u))
+    a = int(np.argmax(z))
+    if z.shape[0] > 1:
+        rest = np.delete(z, a)
+        margin = float(z[a] - np.max(rest))
+    else:
+        margin = float("inf")
+    return a, margin
+
+
+# ----------------------------------------------------------------------------------------
 # Commit / Predict / Refill of Algorithm 1 for one sequence
 # ----------------------------------------------------------------------------------------
 def select_commit_refill(tokens: Sequence[int], filled: Sequence[int], window_len: int,
@@ -315,8 +377,11 @@ def select_commit_refill(tokens: Sequence[int], filled: Sequence[int], window_le
 def step(inp: Dict[str, np.ndarray], *, theta: float, rope_style: int = 0, conf_mode: str,
          tau: float, lam: float, maxprob_thr: float, mask_token_id: int, page_size: int,
          window_len: Optional[np.ndarray] = None, remaining_budget: Optional[np.ndarray] = None,
-         with_attention: bool = True, block_commit: bool = False) -> Dict[str, object]:
-    """All outputs of one decoding step for the arrays of workloads.make_step()."""
+         with_attention: bool = True, block_commit: bool = False, temperature: float = 0.0,
+         sample_seed: Tuple[int, int] = (0, 0)) -> Dict[str, object]:
+    """All outputs of one decoding step for the arrays of workloads.make_step().  With
+    temperature > 0 the token of every mask row is sampled (result key "argmax" then holds the
+    sampled token and "sample_margin" the gap to the runner-up)."""
     filled, prefix_len = inp["filled"], inp["prefix_len"]
     B, W = filled.shape
     ro = reorder(filled, prefix_len, window_len, block_commit)
@@ -331,6 +396,7 @@ def step(inp: Dict[str, np.ndarray], *, theta: float, rope_style: int = 0, conf_
     ent = np.full((B, W), np.nan)
     mp = np.full((B, W), np.nan)
     lse = np.full((B, W), np.nan)
+    margin = np.full((B, W), np.inf)
     per_seq = []
     for b in range(B):
         L = W if window_len is None else int(window_len[b])
@@ -342,6 +408,10 @@ def step(inp: Dict[str, np.ndarray], *, theta: float, rope_style: int = 0, conf_
             ent[b, nf:nf + n_mask] = c["entropy"]
             mp[b, nf:nf + n_mask] = c["maxprob"]
             lse[b, nf:nf + n_mask] = c["lse"]
+            if temperature > 0.0:
+                for i in range(nf, nf + n_mask):
+                    argmax[b, i], margin[b, i] = sample_token(inp["logits"][b, i], temperature, sample_seed, b,
+                                                              int(ro["pos_ids"][b, i]))
         per_seq.append(select_commit_refill(
             inp["window_tokens"][b], filled[b], L, int(prefix_len[b]),
             argmax[b, nf:nf + n_mask], ent[b, nf:nf + n_mask], mp[b, nf:nf + n_mask],
@@ -349,7 +419,7 @@ def step(inp: Dict[str, np.ndarray], *, theta: float, rope_style: int = 0, conf_
             mask_token_id=mask_token_id,
             remaining_budget=None if remaining_budget is None else int(remaining_budget[b]),
             block_commit=block_commit))
-    res.update(argmax=argmax, entropy=ent, maxprob=mp, lse=lse, per_seq=per_seq)
+    res.update(argmax=argmax, entropy=ent, maxprob=mp, lse=lse, per_seq=per_seq, sample_margin=margin)
     return res
 
 
@@ -359,7 +429,8 @@ def step(inp: Dict[str, np.ndarray], *, theta: float, rope_style: int = 0, conf_
 def decode_loop(forward: Callable[[List[int], List[int], List[int]], np.ndarray], *,
                 prefix_len: int, window: int, max_new_tokens: int, conf_mode: str, tau: float,
                 lam: float, maxprob_thr: float, mask_token_id: int,
-                max_steps: int = 100000, block_commit: bool = False) -> Dict[str, object]:
+                max_steps: int = 100000, block_commit: bool = False, temperature: float = 0.0,
+                sample_seed: Tuple[int, int] = (0, 0), seq_index: int = 0) -> Dict[str, object]:
     """Streaming Parallel Decoding (Algorithm 1) for one sequence.
 
     forward(y, tokens_phys, pos_ids) -> logits [W_len, V]: the causal forward of the reordered
@@ -382,6 +453,9 @@ def decode_loop(forward: Callable[[List[int], List[int], List[int]], np.ndarray]
         logits = np.asarray(forward(list(y), [tok[j] for j in perm], [int(p) for p in ro["pos_ids"][0][:L]]))
         n_fwd += L
         c = confidence(logits[nf:L]) if L > nf else dict(argmax=[], entropy=[], maxprob=[])
+        if temperature > 0.0 and L > nf:
+            c["argmax"] = [sample_token(logits[i], temperature, sample_seed, seq_index, int(ro["pos_ids"][0][i]))[0]
+                           for i in range(nf, L)]
         r = select_commit_refill(tok, fil, L, P, c["argmax"], c["entropy"], c["maxprob"],
                                  conf_mode=conf_mode, tau=tau, lam=lam, maxprob_thr=maxprob_thr,
                                  mask_token_id=mask_token_id, remaining_budget=budget, block_commit=block_commit)
