@@ -256,8 +256,8 @@ def confidence(logits_rows: np.ndarray) -> Dict[str, np.ndarray]:
 # A draw from softmax(l / T) is the arg-max over v of l_v / T + g_v with g_v independent standard
 # Gumbel variables (the Gumbel-max identity), g = -ln(-ln u), u uniform on (0, 1).  The uniforms
 # come from a stateless generator so that a row's draw depends only on (seed, sequence index,
-# logical position, token id) and not on how the work is cut up: u = (h >> 8 + 1/2) / 2^24 with h
-# a 32-bit integer hash.  The hash is a xor-shift / odd-multiply finaliser; any implementation has
+# logical position, token id) and not on how the work is cut up: u = ((h >> 9) + 1/2) / 2^23 with h
+# a 32-bit integer hash (23 bits, so that u is also exact in single precision).  The hash is a xor-shift / odd-multiply finaliser; any implementation has
 # to reproduce these integer steps exactly to draw the same tokens.
 _M1 = np.uint32(0x7FEB352D)
 _M2 = np.uint32(0x846CA68B)
@@ -285,10 +285,10 @@ def sample_key(seed_lo: int, seed_hi: int, b: int, pos: int) -> np.uint32:
 
 
 def sample_uniforms(key, V: int) -> np.ndarray:
-    """u_v in (0, 1) for token ids 0..V-1: 24 high bits of mix32(key ^ GOLD * v), centred."""
+    """u_v in (0, 1) for token ids 0..V-1: 23 high bits of mix32(key ^ GOLD * v), centred."""
     with np.errstate(over="ignore"):
         h = mix32(np.uint32(key) ^ (_GOLD * np.arange(V, dtype=np.uint32)))
-    return ((h >> np.uint32(8)).astype(np.float64) + 0.5) * 2.0 ** -24
+    return ((h >> np.uint32(9)).astype(np.float64) + 0.5) * 2.0 ** -23
 
 
 def sample_token(logits_row: np.ndarray, temperature: float, seed: Tuple[int, int], b: int, pos: int) -> Tuple[int, float]:
@@ -380,8 +380,9 @@ def step(inp: Dict[str, np.ndarray], *, theta: float, rope_style: int = 0, conf_
          with_attention: bool = True, block_commit: bool = False, temperature: float = 0.0,
          sample_seed: Tuple[int, int] = (0, 0)) -> Dict[str, object]:
     """All outputs of one decoding step for the arrays of workloads.make_step().  With
-    temperature > 0 the token of every mask row is sampled (result key "argmax" then holds the
-    sampled token and "sample_margin" the gap to the runner-up)."""
+    temperature > 0 the token of every mask row is sampled: "sampled" [B,W] holds the draw of each
+    mask row (-1 elsewhere), "sample_margin" its gap to the runner-up, and the selected slots are
+    filled with the draws; "argmax" stays the greedy arg-max."""
     filled, prefix_len = inp["filled"], inp["prefix_len"]
     B, W = filled.shape
     ro = reorder(filled, prefix_len, window_len, block_commit)
@@ -397,6 +398,7 @@ def step(inp: Dict[str, np.ndarray], *, theta: float, rope_style: int = 0, conf_
     mp = np.full((B, W), np.nan)
     lse = np.full((B, W), np.nan)
     margin = np.full((B, W), np.inf)
+    sampled = np.full((B, W), -1, np.int32)
     per_seq = []
     for b in range(B):
         L = W if window_len is None else int(window_len[b])
@@ -410,16 +412,18 @@ def step(inp: Dict[str, np.ndarray], *, theta: float, rope_style: int = 0, conf_
             lse[b, nf:nf + n_mask] = c["lse"]
             if temperature > 0.0:
                 for i in range(nf, nf + n_mask):
-                    argmax[b, i], margin[b, i] = sample_token(inp["logits"][b, i], temperature, sample_seed, b,
-                                                              int(ro["pos_ids"][b, i]))
+                    sampled[b, i], margin[b, i] = sample_token(inp["logits"][b, i], temperature, sample_seed, b,
+                                                               int(ro["pos_ids"][b, i]))
+        fill_with = sampled if temperature > 0.0 else argmax
         per_seq.append(select_commit_refill(
             inp["window_tokens"][b], filled[b], L, int(prefix_len[b]),
-            argmax[b, nf:nf + n_mask], ent[b, nf:nf + n_mask], mp[b, nf:nf + n_mask],
+            fill_with[b, nf:nf + n_mask], ent[b, nf:nf + n_mask], mp[b, nf:nf + n_mask],
             conf_mode=conf_mode, tau=tau, lam=lam, maxprob_thr=maxprob_thr,
             mask_token_id=mask_token_id,
             remaining_budget=None if remaining_budget is None else int(remaining_budget[b]),
             block_commit=block_commit))
-    res.update(argmax=argmax, entropy=ent, maxprob=mp, lse=lse, per_seq=per_seq, sample_margin=margin)
+    res.update(argmax=argmax, entropy=ent, maxprob=mp, lse=lse, per_seq=per_seq, sampled=sampled,
+               sample_margin=margin)
     return res
 
 

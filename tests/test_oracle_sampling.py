@@ -110,7 +110,7 @@ def test_step_with_temperature_fills_sampled_tokens_and_keeps_confidences():
     greedy = orc.step(inp, **kw)
     hot = orc.step(inp, temperature=5.0, sample_seed=(77, 88), **kw)
     # confidences come from the raw logits either way
-    for key in ("entropy", "maxprob", "lse"):
+    for key in ("entropy", "maxprob", "lse", "argmax"):
         assert np.array_equal(np.nan_to_num(greedy[key], nan=-1.0), np.nan_to_num(hot[key], nan=-1.0))
     differ = 0
     for b in range(cfg.batch):
@@ -118,12 +118,12 @@ def test_step_with_temperature_fills_sampled_tokens_and_keeps_confidences():
         for i in range(nf, cfg.window):
             j = int(hot["perm"][b, i])
             want, _ = orc.sample_token(inp["logits"][b, i], 5.0, (77, 88), b, int(inp["prefix_len"][b]) + j)
-            assert hot["argmax"][b, i] == want
+            assert hot["sampled"][b, i] == want
             differ += int(want != greedy["argmax"][b, i])
         # tau = 50 selects every mask: the window after the step carries exactly the sampled tokens
         r = hot["per_seq"][b]
         n = r["committed_count"]
         for k, j in enumerate(r["mask_slots"]):
             if j >= n:
-                assert r["window_tokens"][j - n] == hot["argmax"][b, nf + k]
+                assert r["window_tokens"][j - n] == hot["sampled"][b, nf + k]
     assert differ > 0            # at T = 5 over ~1000 tokens the draw is essentially never the arg-max everywhere
