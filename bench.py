@@ -198,7 +198,7 @@ class Workload:
     streams (cache, logits) when one copy would fit in L2, and one fresh copy of the small window
     state per iteration."""
 
-    def __init__(self, name, seed, attn_impl, n_state, batch=None):
+    def __init__(self, name, seed, attn_impl, n_state, batch=None, temperature=0.0):
         import torch
         import paper_2512_22737_b200 as w
         from workloads import get_config, make_step
@@ -214,7 +214,7 @@ class Workload:
         self.n_copies = 1 if big > 2 * L2_BYTES else int(np.ceil(3 * L2_BYTES / big)) + 1
         self.c = w.config_for(self.cfg, max_pages_per_seq=inp["block_table"].shape[1],
                               num_pages=inp["k_cache"].shape[0], max_prefix_len=int(inp["prefix_len"].max()),
-                              attn_impl=attn_impl)
+                              attn_impl=attn_impl, sample_temperature=temperature, sample_seed=seed)
         self.step = w.DecodeStep(self.c)
         self.static = {k: w.to_device(inp[k]) for k in ("q", "k", "v", "block_table")}
         self.big = [{k: (w.to_device(inp[k]) if i == 0 else None) for k in ("k_cache", "v_cache", "logits")}
@@ -407,7 +407,7 @@ def run_product(args):
 
     sampler = ClockSampler(local) if rank == 0 else None
     n_state = args.steps + args.warmup
-    wl = Workload(args.workload, rank_seed(rank), args.attn, n_state, args.batch)
+    wl = Workload(args.workload, rank_seed(rank), args.attn, n_state, args.batch, args.temperature)
     if sampler:
         sampler.start()
 
@@ -475,6 +475,7 @@ def run_product(args):
                        "prefix_tokens_per_gpu": int(wl.inp["prefix_len"].sum()), "attn_impl": args.attn,
                        "l2": "inputs_exceed_l2" if wl.n_copies == 1 else f"rotating_{wl.n_copies}_copies",
                        "committed_tokens_per_step": committed_total,
+                       "sample": "argmax" if args.temperature <= 0 else f"gumbel_max_T{args.temperature:g}",
                        "kv_stream_bytes": bts["kv_stream"], "logits_stream_bytes": bts["logits_stream"]},
             "clocks": sampler.summary() if sampler else None,
             "e2e": {"value": e2e_committed / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
@@ -640,6 +641,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing (profiling runs)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling runs)")
+    ap.add_argument("--temperature", type=float, default=0.0,
+                    help="Sample() temperature of the step workloads (0 = arg-max, the headline configuration)")
     ap.add_argument("--loop-batch", type=int, default=16)
     ap.add_argument("--loop-new-tokens", type=int, default=1024)
     ap.add_argument("--loop-windows", type=lambda s: [int(x) for x in s.split(",")], default=[16, 2, 1])

@@ -90,6 +90,9 @@ typedef struct wedlm_config {
   int32_t max_prefix_len;     /* host-known upper bound of prefix_len[b]; sizes the grid   */
   int32_t attn_impl;          /* WEDLM_ATTN_*                                              */
   int32_t commit_mode;        /* WEDLM_COMMIT_*                                            */
+  float   sample_temperature; /* 0: Sample() is the arg-max; > 0: one draw from softmax(l/T) */
+  uint32_t sample_seed_lo;    /* 64-bit seed of the draws, low and high word               */
+  uint32_t sample_seed_hi;
 } wedlm_config_t;
 
 /* Human-readable text of a return code.  Host pointer to a static string. */
@@ -175,7 +178,7 @@ int wedlm_kv_append(const wedlm_config_t* cfg, const void* k, const void* v, con
                     const int32_t* prefix_len, const int32_t* count, int32_t* kv_slot_idx,
                     int32_t* status, void* stream);
 
-/* Bytes of workspace wedlm_confidence_commit needs (uses batch, window, vocab, dtype). */
+/* Bytes of workspace wedlm_confidence_commit needs (uses batch, window, vocab, dtype, sample_temperature). */
 size_t wedlm_confidence_workspace_bytes(const wedlm_config_t* cfg);
 
 /*
@@ -200,6 +203,20 @@ size_t wedlm_confidence_workspace_bytes(const wedlm_config_t* cfg);
  * mask exists, select the single best-scoring mask (leftmost on ties) so that decoding always
  * progresses; write arg-max tokens into the selected slots; shift the window left by n_commit;
  * append fresh masks.
+ *
+ * Sample() at a temperature (Algorithm 1 writes W[i] <- Sample(l_i); Section 6.1 evaluates at 0.1).  With
+ * cfg->sample_temperature = T > 0 every slot filled in this step receives one draw from softmax(l / T)
+ * instead of the arg-max: token = arg-max over v of l_v / T + g_v (lowest v on ties) with Gumbel noise
+ * g_v = -ln(-ln u_v).  The uniforms are stateless, so a draw depends only on (seed, b, logical position,
+ * token id):  mix(x): x ^= x>>16; x *= 0x7FEB352D; x ^= x>>15; x *= 0x846CA68B; x ^= x>>16 (mod 2^32);
+ * key = mix(mix(seed_lo + 0x9E3779B9*b) ^ seed_hi ^ (0x85EBCA6B*pos)), pos = prefix_len[b] + logical slot;
+ * u_v = ((mix(key ^ 0x9E3779B9*v) >> 9) + 0.5) * 2^-23.  Confidences (entropy, max-prob, lse) and the
+ * selection are those of the raw logits; `argmax` reports the draw on the rows filled in this step and the
+ * greedy arg-max on the other mask rows.  Only the selected rows are read a second time; within a row only
+ * tokens whose logit is within 19.6 T of the maximum can win and only they are hashed, so the extra cost
+ * grows with T.  Rows whose logits are all -inf are not supported with T > 0.  Advance the seed (or rely on
+ * the positions advancing) between steps as the application requires; a given (seed, b, pos) always draws
+ * the same noise.  The workspace is larger with T > 0 (wedlm_confidence_workspace_bytes accounts for it).
  */
 int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const int32_t* perm,
                             const int32_t* n_filled, const int32_t* n_commit,
@@ -220,6 +237,8 @@ int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const
  *   tilt_ids      in  i32  [B,W] or NULL: the logit of token tilt_ids[b,i] of physical row i gets +tilt
  *                 (the additive tilt toward a target sequence of the end-to-end configuration); -1 = none
  *   all other arguments as in wedlm_confidence_commit; statistics come from fp32 logits (not rounded to bf16).
+ *   cfg->sample_temperature must be 0 (the logits are never stored, so there is nothing to draw from after the
+ *   selection): WEDLM_ERR_UNSUPPORTED otherwise.
  * Workspace: wedlm_lmhead_confidence_workspace_bytes(cfg) = batch*window*ceil(vocab/128)*16 bytes (an upper
  * bound: the vocabulary tile width, 128..256, is chosen per launch).
  */

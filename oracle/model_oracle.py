@@ -71,8 +71,10 @@ def forward_window(weights: Dict[str, np.ndarray], mcfg, committed: Sequence[int
 
 def decode(weights, mcfg, prompt: Sequence[int], target: Sequence[int], *, tilt: float, window: int,
            max_new_tokens: int, conf_mode: str, tau: float, lam: float, maxprob_thr: float,
-           block_commit: bool = False) -> Dict[str, object]:
-    """Algorithm 1 for one sequence on the model above; logits[row, target[position of row]] += tilt."""
+           block_commit: bool = False, temperature: float = 0.0, sample_seed=(0, 0),
+           seq_index: int = 0) -> Dict[str, object]:
+    """Algorithm 1 for one sequence on the model above; logits[row, target[position of row]] += tilt.
+    With temperature > 0 the filled tokens are draws (keyed by sample_seed, seq_index and position)."""
     prompt = [int(t) for t in prompt]
 
     def forward(y: List[int], toks: List[int], pos: List[int]) -> np.ndarray:
@@ -84,4 +86,5 @@ def decode(weights, mcfg, prompt: Sequence[int], target: Sequence[int], *, tilt:
 
     return orc.decode_loop(forward, prefix_len=len(prompt), window=window, max_new_tokens=max_new_tokens,
                            conf_mode=conf_mode, tau=tau, lam=lam, maxprob_thr=maxprob_thr,
-                           mask_token_id=mcfg.mask_token_id, block_commit=block_commit)
+                           mask_token_id=mcfg.mask_token_id, block_commit=block_commit, temperature=temperature,
+                           sample_seed=sample_seed, seq_index=seq_index)

@@ -41,6 +41,7 @@ class WedlmConfig(ctypes.Structure):
         ("softmax_scale", ctypes.c_float), ("conf_mode", ctypes.c_int32), ("tau", ctypes.c_float),
         ("lambda_", ctypes.c_float), ("maxprob_thr", ctypes.c_float), ("mask_token_id", ctypes.c_int32),
         ("max_prefix_len", ctypes.c_int32), ("attn_impl", ctypes.c_int32), ("commit_mode", ctypes.c_int32),
+        ("sample_temperature", ctypes.c_float), ("sample_seed_lo", ctypes.c_uint32), ("sample_seed_hi", ctypes.c_uint32),
     ]
 
     @property
@@ -138,7 +139,7 @@ def make_config(*, batch, window, n_q_heads=1, n_kv_heads=1, head_dim=128, page_
                 max_pages_per_seq=1, num_pages=1, vocab=1, dtype="bf16", rope_style=0,
                 rope_theta=1.0e6, softmax_scale=0.0, conf_mode="entropy", tau=0.3, lam=0.1,
                 maxprob_thr=0.9, mask_token_id=0, max_prefix_len=0, attn_impl="auto",
-                commit_mode="streaming") -> WedlmConfig:
+                commit_mode="streaming", sample_temperature=0.0, sample_seed=0) -> WedlmConfig:
     c = WedlmConfig()
     c.batch, c.window, c.n_q_heads, c.n_kv_heads, c.head_dim = batch, window, n_q_heads, n_kv_heads, head_dim
     c.page_size, c.max_pages_per_seq, c.num_pages, c.vocab = page_size, max_pages_per_seq, num_pages, vocab
@@ -149,6 +150,8 @@ def make_config(*, batch, window, n_q_heads=1, n_kv_heads=1, head_dim=128, page_
     c.max_prefix_len = max_prefix_len
     c.attn_impl = {"auto": WEDLM_ATTN_AUTO, "generic": WEDLM_ATTN_GENERIC, "tensor": WEDLM_ATTN_TENSOR}[attn_impl]
     c.commit_mode = {"streaming": 0, "block": 1}[commit_mode]
+    c.sample_temperature = sample_temperature
+    c.sample_seed_lo, c.sample_seed_hi = sample_seed & 0xFFFFFFFF, (sample_seed >> 32) & 0xFFFFFFFF
     return c
 
 
@@ -362,7 +365,8 @@ class DecodeStep:
 
 
 def config_for(step_cfg, *, max_pages_per_seq: int, num_pages: int, max_prefix_len: int,
-               attn_impl: str = "auto", batch: Optional[int] = None, commit_mode: str = "streaming") -> WedlmConfig:
+               attn_impl: str = "auto", batch: Optional[int] = None, commit_mode: str = "streaming",
+               sample_temperature: float = 0.0, sample_seed: int = 0) -> WedlmConfig:
     """wedlm_config_t for an object with the attribute names of a workload description
     (batch, window, n_q_heads, n_kv_heads, head_dim, page_size, vocab, dtype, rope_theta,
     conf_mode, tau, lam, maxprob_thr, mask_token_id)."""
@@ -373,4 +377,4 @@ def config_for(step_cfg, *, max_pages_per_seq: int, num_pages: int, max_prefix_l
         vocab=step_cfg.vocab, dtype=step_cfg.dtype, rope_theta=step_cfg.rope_theta,
         conf_mode=step_cfg.conf_mode, tau=step_cfg.tau, lam=step_cfg.lam, maxprob_thr=step_cfg.maxprob_thr,
         mask_token_id=step_cfg.mask_token_id, max_prefix_len=max_prefix_len, attn_impl=attn_impl,
-        commit_mode=commit_mode)
+        commit_mode=commit_mode, sample_temperature=sample_temperature, sample_seed=sample_seed)

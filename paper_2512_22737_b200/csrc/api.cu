@@ -43,6 +43,7 @@ int check_config(const wedlm_config_t* c, bool need_cache, bool need_vocab) {
     if (c->vocab < 1) return WEDLM_ERR_INVALID_ARG;
     if (c->conf_mode != WEDLM_CONF_ENTROPY && c->conf_mode != WEDLM_CONF_MAXPROB) return WEDLM_ERR_INVALID_ARG;
     if (c->tau != c->tau || c->lambda != c->lambda || c->maxprob_thr != c->maxprob_thr) return WEDLM_ERR_INVALID_ARG;
+    if (!(c->sample_temperature >= 0.f) || c->sample_temperature > 3.0e38f) return WEDLM_ERR_INVALID_ARG;
   }
   return WEDLM_OK;
 }
@@ -260,6 +261,7 @@ int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, co
   int rc = check_config(cfg, false, true);
   if (rc != WEDLM_OK) return rc;
   if (cfg->dtype != WEDLM_DTYPE_BF16 || hidden < 64 || hidden % 64 != 0) return WEDLM_ERR_UNSUPPORTED;
+  if (cfg->sample_temperature > 0.f) return WEDLM_ERR_UNSUPPORTED;     // no stored logits to draw from
   if ((long long)cfg->batch * cfg->window >= (1ll << 31) / 2) return WEDLM_ERR_UNSUPPORTED;
   if (cfg->batch == 0) return WEDLM_OK;
   if (!hidden_states || !lm_head || !perm || !n_filled || !n_commit || !window_tokens || !filled || !prefix_len || !workspace)

@@ -88,7 +88,7 @@ int launch_conf_commit(const Shape& s, const wedlm_config_t* cfg, int n_chunks, 
                        const int32_t* n_filled, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
                        int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget, int32_t* argmax,
                        float* maxprob, float* entropy, float* lse, int32_t* committed_tokens, int32_t* committed_count,
-                       int32_t* filled_count, cudaStream_t st);
+                       int32_t* filled_count, cudaStream_t st, void* sample_ws = nullptr);
 
 // Fused LM head + confidence pass 1: partials [B*W][n_tiles] (n_tiles <= ceil(V/128), returned) from hidden states and the output embedding.
 int lmhead_conf_tiles(int vocab);

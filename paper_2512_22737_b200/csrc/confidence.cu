@@ -6,6 +6,10 @@
 // s = sum e^(x-m), t = sum (x-m) e^(x-m).  Pass 2 (conf_commit_kernel, one warp per sequence)
 // merges the chunks of every row in double precision, lse = m + ln s, p_max = 1/s,
 // H = ln s - t/s, then runs the window update.
+//
+// Sample() at a temperature T > 0 (Algorithm 1, "W[i] <- Sample(l_i)") is a third pass over the rows that
+// pass 2 selected, and only those: sample_fill_kernel draws token = arg-max_v (l_v - m) / T + g_v with
+// Gumbel noise from a stateless hash of (seed, sequence, position, token) and overwrites the greedy token.
 #include <math_constants.h>
 
 #include "common.cuh"
@@ -402,7 +406,49 @@ __device__ void commit_shift_refill(int b, int W, int L, int n, const int* tok_s
 struct ConfParams {
   int W, n_chunks, conf_mode, mask_id;
   float tau, lambda, thr;
+  float temperature;            // 0: greedy
+  uint32_t seed_lo, seed_hi;
 };
+
+// Scratch of the sampling pass, carved from the caller's workspace behind the chunk partials.
+struct SampleWs {
+  unsigned long long* best;     // [rows] packed (ordered score bits, ~token): merged with atomicMax
+  float2* cm;                   // [rows] (cut-off logit below which a token cannot win, row maximum)
+  int* sel_row;                 // [n_sel] rows selected in this step, any order
+  uint32_t* key;                // [rows] hash key of the row
+  int* dst;                     // [rows] index into window_tokens of the slot after the shift, or -1
+  int* cnt;                     // [rows] chunks finished
+  int* n_sel;                   // [1]
+};
+constexpr size_t kSampleWsPerRow = 8 + 8 + 4 + 4 + 4 + 4;
+constexpr size_t kSampleWsFixed = 16;
+
+__host__ inline SampleWs carve_sample_ws(void* base, size_t rows) {
+  SampleWs w;
+  unsigned char* p = reinterpret_cast<unsigned char*>(base);
+  w.best = reinterpret_cast<unsigned long long*>(p); p += rows * 8;
+  w.cm = reinterpret_cast<float2*>(p);               p += rows * 8;
+  w.sel_row = reinterpret_cast<int*>(p);             p += rows * 4;
+  w.key = reinterpret_cast<uint32_t*>(p);            p += rows * 4;
+  w.dst = reinterpret_cast<int*>(p);                 p += rows * 4;
+  w.cnt = reinterpret_cast<int*>(p);                 p += rows * 4;
+  w.n_sel = reinterpret_cast<int*>(p);
+  return w;
+}
+
+// Stateless uniforms of the sampler: a bijective 32-bit finaliser (xor-shift / odd multiply).
+__device__ __forceinline__ uint32_t mix32(uint32_t x) {
+  x ^= x >> 16; x *= 0x7FEB352Du;
+  x ^= x >> 15; x *= 0x846CA68Bu;
+  x ^= x >> 16;
+  return x;
+}
+__device__ __forceinline__ uint32_t sample_row_key(uint32_t seed_lo, uint32_t seed_hi, uint32_t b, uint32_t pos) {
+  return mix32(mix32(seed_lo + 0x9E3779B9u * b) ^ seed_hi ^ (0x85EBCA6Bu * pos));
+}
+// Range of the noise g = -ln(-ln u) for u = (k + 1/2) 2^-23, k < 2^23: [-2.812, 16.636].  A token can only win
+// against the row's arg-max (score >= m/T - 2.812) if its logit is within (16.636 + 2.812) T of the maximum.
+constexpr float kGumbelSpan = 19.6f;
 
 // One block per sequence with up to one warp per window row.  Each warp merges the chunk partials of
 // whole rows (lanes over chunks, double precision), then warp 0 runs the selection and the window update.
@@ -411,13 +457,14 @@ conf_commit_kernel(ConfParams p, const float4* __restrict__ part, const int32_t*
                    const int32_t* __restrict__ n_filled, const int32_t* __restrict__ n_commit,
                    int32_t* window_tokens, uint8_t* filled, int32_t* prefix_len, int32_t* window_len,
                    int32_t* remaining_budget, int32_t* argmax, float* maxprob, float* entropy, float* lse,
-                   int32_t* committed_tokens, int32_t* committed_count, int32_t* filled_count) {
+                   int32_t* committed_tokens, int32_t* committed_count, int32_t* filled_count, SampleWs sw) {
   extern __shared__ unsigned char sm_raw[];
   const int W = p.W;
   double* score = reinterpret_cast<double*>(sm_raw);        // [W] per mask k
   int* am = reinterpret_cast<int*>(score + W);                // [W] arg-max per mask k
   int* tok_s = am + W;                                        // [W] logical
-  uint8_t* fil_s = reinterpret_cast<uint8_t*>(tok_s + W);     // [W] logical
+  float* mrow = reinterpret_cast<float*>(tok_s + W);          // [W] row maximum per mask k
+  uint8_t* fil_s = reinterpret_cast<uint8_t*>(mrow + W);      // [W] logical
   uint8_t* pass = fil_s + W;                                  // [W] per mask k
 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -495,6 +542,7 @@ conf_commit_kernel(ConfParams p, const float4* __restrict__ part, const int32_t*
       }
       score[k] = sc;
       am[k] = a;
+      mrow[k] = m;
       pass[k] = ok ? 1 : 0;
     }
   }
@@ -522,17 +570,103 @@ conf_commit_kernel(ConfParams p, const float4* __restrict__ part, const int32_t*
     n_pass = 1;
   }
   __syncwarp();
+  const int P0 = prefix_len[b];                               // before the commit below moves it
+  const int n_drop = min(max(n_commit[b], 0), L);
   for (int k = lane; k < n_mask; k += 32) {
     if (pass[k]) {
       const int j = perm[o + nf + k];
       tok_s[j] = am[k];
       fil_s[j] = 1;
+      if (p.temperature > 0.f) {                              // hand the row to the sampling pass
+        const size_t row = o + nf + k;
+        sw.sel_row[atomicAdd(sw.n_sel, 1)] = (int)row;
+        sw.key[row] = sample_row_key(p.seed_lo, p.seed_hi, (uint32_t)b, (uint32_t)(P0 + j));
+        sw.dst[row] = j >= n_drop ? (int)(o + j - n_drop) : -1;
+        sw.cm[row] = make_float2(mrow[k] - p.temperature * kGumbelSpan, mrow[k]);
+        sw.cnt[row] = 0;
+        sw.best[row] = 0ull;
+      }
     }
   }
   if (lane == 0 && filled_count) filled_count[b] = n_pass;
   __syncwarp();
   commit_shift_refill(b, W, L, n_commit[b], tok_s, fil_s, p.mask_id, window_tokens, filled, prefix_len, window_len,
                       remaining_budget, committed_tokens, committed_count);
+}
+
+// Sampling pass: persistent blocks over (selected row, chunk).  Every chunk offers its best perturbed score
+// to the row's packed maximum; the block that finishes a row last writes the drawn token into the window.
+__device__ __forceinline__ unsigned long long pack_score(float z, int idx) {
+  uint32_t bits = __float_as_uint(z);
+  bits = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);          // order-preserving map to unsigned
+  return ((unsigned long long)bits << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)idx);   // equal scores: lower token
+}
+
+template <typename T, bool VEC>
+__global__ void __launch_bounds__(kConfThreads)
+sample_fill_kernel(int V, int n_chunks, float inv_t, const T* __restrict__ logits, SampleWs sw,
+                   int32_t* __restrict__ argmax, int32_t* __restrict__ window_tokens) {
+  constexpr int VL = VecTraits<T>::VL;
+  constexpr int CHUNK = conf_chunk_elems<T>();
+  const int tid = threadIdx.x, lane = tid & 31;
+  const long long n_items = (long long)(*sw.n_sel) * n_chunks;
+  for (long long it = blockIdx.x; it < n_items; it += gridDim.x) {
+    const int r = (int)(it / n_chunks), chunk = (int)(it - (long long)r * n_chunks);
+    const int row = sw.sel_row[r];
+    const uint32_t key = sw.key[row];
+    const float2 cm = sw.cm[row];
+    const T* src = logits + (size_t)row * V;
+    const int base = chunk * CHUNK;
+    float bz = -CUDART_INF_F;
+    int bi = 0x7fffffff;
+    auto consider = [&](float x, int idx) {
+      if (x >= cm.x) {                                                   // few tokens get here unless T is large
+        const uint32_t h = mix32(key ^ (0x9E3779B9u * (uint32_t)idx));
+        const float u = ((float)(h >> 9) + 0.5f) * 1.1920928955078125e-07f;   // exact: 24 significant bits
+        const float g = -logf(-logf(u));
+        const float z = fmaf(x - cm.y, inv_t, g);
+        if (z > bz || (z == bz && idx < bi)) { bz = z; bi = idx; }
+      }
+    };
+#pragma unroll
+    for (int k = 0; k < kConfVecs; ++k) {
+      const int e0 = base + (k * kConfThreads + tid) * VL;
+      if (VEC) {
+        if (e0 < V) {                                                    // V % VL == 0 on this path
+          const uint4 raw = __ldg(reinterpret_cast<const uint4*>(src + e0));
+          float xv[VL];
+          unpack16(raw, xv);
+#pragma unroll
+          for (int e = 0; e < VL; ++e) consider(xv[e], e0 + e);
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < VL; ++e)
+          if (e0 + e < V) consider(ld_as_float(src, e0 + e), e0 + e);
+      }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float oz = __shfl_xor_sync(0xffffffffu, bz, off);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+      if (oz > bz || (oz == bz && oi < bi)) { bz = oz; bi = oi; }
+    }
+    if (lane == 0 && bi != 0x7fffffff) atomicMax(sw.best + row, pack_score(bz, bi));
+    __syncthreads();                                                     // every warp has made its offer
+    if (tid == 0) {
+      __threadfence();
+      if (atomicAdd(sw.cnt + row, 1) == n_chunks - 1) {                  // this block completes the row
+        __threadfence();
+        const unsigned long long bb = atomicMax(sw.best + row, 0ull);    // coherent read
+        if (bb != 0ull) {
+          const int tok = (int)(0xFFFFFFFFu - (uint32_t)(bb & 0xFFFFFFFFull));
+          if (argmax) argmax[row] = tok;
+          const int d = sw.dst[row];
+          if (d >= 0) window_tokens[d] = tok;
+        }
+      }
+    }
+  }
 }
 
 __global__ void __launch_bounds__(32)
@@ -560,7 +694,10 @@ static int conf_chunks(const wedlm_config_t* cfg) {
 }
 
 size_t confidence_workspace_bytes(const wedlm_config_t* cfg) {
-  return (size_t)cfg->batch * cfg->window * conf_chunks(cfg) * sizeof(float4);
+  const size_t rows = (size_t)cfg->batch * cfg->window;
+  size_t bytes = rows * conf_chunks(cfg) * sizeof(float4);
+  if (cfg->sample_temperature > 0.f) bytes += rows * kSampleWsPerRow + kSampleWsFixed;
+  return bytes;
 }
 
 int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* logits, const int32_t* perm,
@@ -604,25 +741,56 @@ int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* log
   }
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return WEDLM_ERR_CUDA;
-  return launch_conf_commit(s, cfg, n_chunks, part, perm, n_filled, n_commit, window_tokens, filled, prefix_len, window_len,
-                            remaining_budget, argmax, maxprob, entropy, lse, committed_tokens, committed_count,
-                            filled_count, st);
+  const bool sampling = cfg->sample_temperature > 0.f;
+  const size_t rows = (size_t)s.B * s.W;
+  void* sample_ws = sampling ? reinterpret_cast<unsigned char*>(workspace) + rows * n_chunks * sizeof(float4) : nullptr;
+  int rc = launch_conf_commit(s, cfg, n_chunks, part, perm, n_filled, n_commit, window_tokens, filled, prefix_len, window_len,
+                              remaining_budget, argmax, maxprob, entropy, lse, committed_tokens, committed_count,
+                              filled_count, st, sample_ws);
+  if (rc != WEDLM_OK || !sampling) return rc;
+  // third pass: draw the tokens of the rows selected above
+  const SampleWs sw = carve_sample_ws(sample_ws, rows);
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  long long grid = (long long)sms * 8;
+  if (grid > blocks) grid = blocks;
+  const float inv_t = (float)(1.0 / (double)cfg->sample_temperature);
+  if (s.dtype == WEDLM_DTYPE_BF16) {
+    using T = __nv_bfloat16;
+    const bool vec = (s.V % VecTraits<T>::VL == 0) && ((uintptr_t)logits % 16 == 0);
+    if (vec) sample_fill_kernel<T, true><<<(unsigned)grid, kConfThreads, 0, st>>>(s.V, n_chunks, inv_t, (const T*)logits, sw, argmax, window_tokens);
+    else     sample_fill_kernel<T, false><<<(unsigned)grid, kConfThreads, 0, st>>>(s.V, n_chunks, inv_t, (const T*)logits, sw, argmax, window_tokens);
+  } else {
+    using T = float;
+    const bool vec = (s.V % VecTraits<T>::VL == 0) && ((uintptr_t)logits % 16 == 0);
+    if (vec) sample_fill_kernel<T, true><<<(unsigned)grid, kConfThreads, 0, st>>>(s.V, n_chunks, inv_t, (const T*)logits, sw, argmax, window_tokens);
+    else     sample_fill_kernel<T, false><<<(unsigned)grid, kConfThreads, 0, st>>>(s.V, n_chunks, inv_t, (const T*)logits, sw, argmax, window_tokens);
+  }
+  count_launch();
+  return cuda_ok(cudaGetLastError());
 }
 
-// Pass 2 alone: merge `n_chunks` partials (m, s, t, argmax) per mask row, select, commit, refill.
+// Pass 2 alone: merge `n_chunks` partials (m, s, t, argmax) per mask row, select, commit, refill.  With a
+// sampling scratch it also lists the selected rows for sample_fill_kernel.
 int launch_conf_commit(const Shape& s, const wedlm_config_t* cfg, int n_chunks, const void* partials, const int32_t* perm,
                        const int32_t* n_filled, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
                        int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget, int32_t* argmax,
                        float* maxprob, float* entropy, float* lse, int32_t* committed_tokens, int32_t* committed_count,
-                       int32_t* filled_count, cudaStream_t st) {
-  ConfParams p{s.W, n_chunks, cfg->conf_mode, cfg->mask_token_id, cfg->tau, cfg->lambda, cfg->maxprob_thr};
-  size_t smem = (size_t)s.W * (sizeof(double) + 2 * sizeof(int) + 2);
+                       int32_t* filled_count, cudaStream_t st, void* sample_ws) {
+  ConfParams p{s.W, n_chunks, cfg->conf_mode, cfg->mask_token_id, cfg->tau, cfg->lambda, cfg->maxprob_thr,
+               sample_ws ? cfg->sample_temperature : 0.f, cfg->sample_seed_lo, cfg->sample_seed_hi};
+  SampleWs sw{};
+  if (sample_ws) {
+    sw = carve_sample_ws(sample_ws, (size_t)s.B * s.W);
+    if (cudaMemsetAsync(sw.n_sel, 0, sizeof(int), st) != cudaSuccess) return WEDLM_ERR_CUDA;
+  }
+  size_t smem = (size_t)s.W * (sizeof(double) + 2 * sizeof(int) + sizeof(float) + 2);
   int commit_threads = 32 * s.W;
   commit_threads = commit_threads < 128 ? 128 : (commit_threads > 1024 ? 1024 : commit_threads);
   conf_commit_kernel<<<s.B, commit_threads, smem, st>>>(p, reinterpret_cast<const float4*>(partials), perm, n_filled, n_commit,
                                                         window_tokens, filled, prefix_len, window_len, remaining_budget,
                                                         argmax, maxprob, entropy, lse, committed_tokens, committed_count,
-                                                        filled_count);
+                                                        filled_count, sw);
   count_launch();
   return cuda_ok(cudaGetLastError());
 }

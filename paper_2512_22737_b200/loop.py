@@ -28,7 +28,7 @@ class StreamingDecoder:
                  conf_mode: str = "entropy", tau: float = 0.3, lam: float = 0.1, maxprob_thr: float = 0.9,
                  tilt: float = 0.0, target: Optional[np.ndarray] = None, page_size: int = 16,
                  attn_impl: str = "auto", seed: int = 0, commit_mode: str = "streaming",
-                 fused_lm_head: bool = False):
+                 fused_lm_head: bool = False, temperature: float = 0.0, sample_seed: int = 0):
         self.m = mcfg
         self.B, self.W = batch, window
         self.dtype = torch.bfloat16 if mcfg.dtype == "bf16" else torch.float32
@@ -49,7 +49,9 @@ class StreamingDecoder:
             page_size=page_size, max_pages_per_seq=pages_per_seq, num_pages=self.num_pages, vocab=mcfg.vocab,
             dtype=mcfg.dtype, rope_theta=mcfg.rope_theta, conf_mode=conf_mode, tau=tau, lam=lam,
             maxprob_thr=maxprob_thr, mask_token_id=mcfg.mask_token_id, max_prefix_len=max_total_len,
-            attn_impl=attn_impl, commit_mode=commit_mode)
+            attn_impl=attn_impl, commit_mode=commit_mode, sample_temperature=temperature, sample_seed=sample_seed)
+        if fused_lm_head and temperature > 0.0:
+            raise ValueError("the fused LM head keeps no logits to sample from; use fused_lm_head=False with a temperature")
         self.step_bufs = w.DecodeStep(self.cfg)
         # fused LM head: logits are never materialised; the output embedding is kept as [V, H]
         self.fused_lm_head = fused_lm_head

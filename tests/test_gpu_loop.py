@@ -45,6 +45,32 @@ def test_tiny_model_text_is_token_exact(W, tilt, tau):
         assert got["steps"] < N
 
 
+@pytest.mark.parametrize("W,tilt,tau,T", [(4, 6.0, 0.5, 0.7), (8, 4.0, 2.0, 1.0), (8, 8.0, 0.35, 0.1), (1, 2.0, 0.3, 1.5)])
+def test_tiny_model_sampled_text_is_token_exact(W, tilt, tau, T):
+    """Sample() at a temperature: the GPU loop and the oracle draw from the same counter-based generator, keyed
+    by (seed, sequence, position), so the sampled text agrees token by token as well."""
+    from paper_2512_22737_b200.loop import StreamingDecoder
+    B, P, N = 3, 21, 26
+    seed = (3 << 32) | 77
+    wts = make_model(TINY)
+    pt = make_prompts_and_targets(TINY, B, P, N)
+    dec = StreamingDecoder(TINY, wts, batch=B, window=W, max_total_len=P + N, tau=tau, lam=0.1, tilt=tilt,
+                           target=pt["target"], temperature=T, sample_seed=seed)
+    dec.prefill(pt["prompt"])
+    got = dec.generate(N)
+    greedy_same = 0
+    for b in range(B):
+        ref = mo.decode(wts, TINY, pt["prompt"][b], pt["target"][b], tilt=tilt, window=W, max_new_tokens=N,
+                        conf_mode="entropy", tau=tau, lam=0.1, maxprob_thr=0.9, temperature=T,
+                        sample_seed=(seed & 0xFFFFFFFF, seed >> 32), seq_index=b)
+        assert got["y"][b] == ref["y"], (b, got["y"][b], ref["y"])
+        greedy = mo.decode(wts, TINY, pt["prompt"][b], pt["target"][b], tilt=tilt, window=W, max_new_tokens=N,
+                           conf_mode="entropy", tau=tau, lam=0.1, maxprob_thr=0.9)
+        greedy_same += int(greedy["y"] == ref["y"])
+    if T >= 0.7:
+        assert greedy_same < B          # the sampled text is not the greedy text
+
+
 @pytest.mark.parametrize("W,tilt,tau", [(4, 8.0, 0.5), (8, 30.0, 0.35)])
 def test_tiny_model_block_wise_baseline_is_token_exact(W, tilt, tau):
     from paper_2512_22737_b200.loop import StreamingDecoder

@@ -1,0 +1,165 @@
+"""GPU-vs-oracle parity of Sample() at a temperature (Algorithm 1, "W[i] <- Sample(l_i)").
+
+The draw is an integer decided by floating point: both sides take arg-max of l/T + Gumbel noise from
+the same counter-based generator, the oracle in fp64 and the kernel in fp32.  Rows whose winning margin
+(in the oracle) is inside the tie band are excluded and counted; everything else must match exactly."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2512_22737_b200 as w
+from workloads import get_config, make_step
+from oracle import wedlm_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+SAMPLE_TIE_BAND = 1e-3       # on the perturbed score l/T + g
+
+
+def _run(cfg, inp, T, seed, window_len=None, budget=None, commit_mode="streaming"):
+    d = {k: w.to_device(v) for k, v in inp.items() if k in ("filled", "window_tokens", "prefix_len", "logits")}
+    c = w.config_for(cfg, max_pages_per_seq=inp["block_table"].shape[1], num_pages=inp["k_cache"].shape[0],
+                     max_prefix_len=int(inp["prefix_len"].max()), batch=inp["filled"].shape[0],
+                     commit_mode=commit_mode, sample_temperature=T, sample_seed=seed)
+    step = w.DecodeStep(c)
+    wl = None if window_len is None else torch.tensor(window_len, dtype=torch.int32, device="cuda")
+    rb = None if budget is None else torch.tensor(budget, dtype=torch.int32, device="cuda")
+    step.reorder(d["filled"], d["window_tokens"], d["prefix_len"], wl)
+    step.confidence_commit(d["logits"], d["window_tokens"], d["filled"], d["prefix_len"], wl, rb)
+    torch.cuda.synchronize()
+    ref = orc.step(inp, theta=cfg.rope_theta, conf_mode=cfg.conf_mode, tau=cfg.tau, lam=cfg.lam,
+                   maxprob_thr=cfg.maxprob_thr, mask_token_id=cfg.mask_token_id, page_size=cfg.page_size,
+                   window_len=window_len, remaining_budget=budget, with_attention=False,
+                   block_commit=(commit_mode == "block"), temperature=T,
+                   sample_seed=(seed & 0xFFFFFFFF, seed >> 32))
+    return step, d, ref
+
+
+def _compare(cfg, inp, step, d, ref, tau_band=1e-3):
+    """Returns (rows compared, rows excluded for a near-tie of the draw, draws that differ from greedy)."""
+    B, W = inp["filled"].shape
+    am = step.argmax.cpu().numpy()
+    tok = d["window_tokens"].cpu().numpy()
+    fil = d["filled"].cpu().numpy()
+    fc = step.filled_count.cpu().numpy()
+    compared = excluded = nongreedy = 0
+    for b in range(B):
+        ps = ref["per_seq"][b]
+        sc = np.asarray(ps["scores"], dtype=np.float64)
+        thr = cfg.tau if cfg.conf_mode == "entropy" else -cfg.maxprob_thr
+        if len(sc) and np.isfinite(thr) and (np.abs(sc - thr) <= tau_band * max(1.0, abs(thr))).any():
+            continue                                   # selection itself inside the tie band: covered elsewhere
+        if len(sc) > 1 and not (sc <= thr).any():
+            srt = np.sort(sc)
+            if srt[1] - srt[0] <= tau_band * max(1.0, abs(srt[0])):
+                continue
+        assert fc[b] == ps["filled_count"]
+        assert fil[b].tolist() == ps["filled"]
+        nf = int(ref["n_filled"][b])
+        n = ps["committed_count"]
+        want_tok = list(ps["window_tokens"])
+        chosen = set(ps["filled_slots"])
+        for k, j in enumerate(ps["mask_slots"]):
+            i = nf + k
+            if j in chosen:
+                if ref["sample_margin"][b, i] < SAMPLE_TIE_BAND:
+                    excluded += 1
+                    want_tok[j - n] = int(tok[b, j - n])       # either candidate is acceptable here
+                    continue
+                compared += 1
+                assert am[b, i] == ref["sampled"][b, i], (b, i, am[b, i], ref["sampled"][b, i], ref["sample_margin"][b, i])
+                nongreedy += int(ref["sampled"][b, i] != ref["argmax"][b, i])
+            else:
+                assert am[b, i] == ref["argmax"][b, i]          # rows not filled keep the greedy statistic
+        assert tok[b].tolist() == want_tok, (b, tok[b].tolist(), want_tok)
+    return compared, excluded, nongreedy
+
+
+@pytest.mark.parametrize("T", [0.1, 1.0, 4.0])
+@pytest.mark.parametrize("seed", [1, (7 << 32) | 123456789])
+def test_cfg1_tiny_fp32_every_mask_selected(T, seed):
+    cfg = get_config("cfg1_tiny").replace(conf_mode="entropy", tau=50.0)   # every mask is filled: many draws per step
+    total = 0
+    for s in (3, 4):
+        inp = make_step(cfg, seed=s)
+        step, d, ref = _run(cfg, inp, T, seed)
+        c, e, ng = _compare(cfg, inp, step, d, ref)
+        total += c
+        assert e <= 1
+        if T >= 1.0:
+            assert ng > 0                                       # the draw really is not the arg-max
+    assert total >= 8, total
+
+
+@pytest.mark.parametrize("T", [0.1, 0.7, 3.0])
+def test_bf16_full_vocabulary_rows(T):
+    """V = 151936 spans 19 chunks with a ragged last one; T = 3 sends nearly every token through the hash."""
+    cfg = get_config("cfg2_qwen_b1").replace(tau=50.0)
+    inp = make_step(cfg, seed=5)
+    step, d, ref = _run(cfg, inp, T, 99)
+    c, e, ng = _compare(cfg, inp, step, d, ref)
+    assert c >= 4 and e <= 1
+    if T >= 0.7:
+        assert ng > 0
+
+
+def test_threshold_selection_with_boosts_and_paper_temperature():
+    cfg = get_config("cfg2_qwen_b1").replace(vocab=20000, batch=6, boost=14.0, boost_prob=0.6, name="mixed")
+    seen = 0
+    for s in (11, 12, 13):
+        inp = make_step(cfg, seed=s)
+        step, d, ref = _run(cfg, inp, 0.1, 2024)
+        c, e, _ = _compare(cfg, inp, step, d, ref)
+        seen += c
+    assert seen >= 6
+
+
+def test_unaligned_vocab_short_windows_budget_and_block_mode():
+    cfg = get_config("cfg2_qwen_b1").replace(vocab=10007, batch=4, window=8, tau=50.0, name="oddvocab")
+    inp = make_step(cfg, seed=21)
+    wl = np.array([8, 5, 1, 0], np.int32)
+    rb = np.array([3, 0, 9, 2], np.int32)
+    step, d, ref = _run(cfg, inp, 1.5, 31337, window_len=wl, budget=rb)
+    c, e, _ = _compare(cfg, inp, step, d, ref)
+    assert c >= 3
+    step, d, ref = _run(cfg, inp, 1.5, 31337, commit_mode="block")
+    _compare(cfg, inp, step, d, ref)
+
+
+def test_same_seed_same_draw_other_seed_other_draw_and_greedy_when_off():
+    cfg = get_config("cfg2_qwen_b1").replace(vocab=32000, batch=3, tau=50.0, name="seeds")
+    inp = make_step(cfg, seed=8)
+    a, da, _ = _run(cfg, inp, 2.0, 5)
+    b, db, _ = _run(cfg, inp, 2.0, 5)
+    c, dc, _ = _run(cfg, inp, 2.0, 6)
+    g, dg, ref = _run(cfg, inp, 0.0, 5)
+    assert torch.equal(da["window_tokens"], db["window_tokens"])
+    assert not torch.equal(da["window_tokens"], dc["window_tokens"])
+    np.testing.assert_array_equal(g.argmax.cpu().numpy(), ref["argmax"])
+    for bb in range(cfg.batch):
+        assert dg["window_tokens"][bb].cpu().tolist() == ref["per_seq"][bb]["window_tokens"]
+
+
+def test_fused_lm_head_refuses_sampling_and_workspace_grows():
+    cfg = get_config("cfg2_qwen_b1")
+    c0 = w.config_for(cfg, max_pages_per_seq=8, num_pages=8, max_prefix_len=64)
+    c1 = w.config_for(cfg, max_pages_per_seq=8, num_pages=8, max_prefix_len=64, sample_temperature=0.1)
+    assert w.wedlm_confidence_workspace_bytes(c1) > w.wedlm_confidence_workspace_bytes(c0)
+    bad = w.config_for(cfg, max_pages_per_seq=8, num_pages=8, max_prefix_len=64, sample_temperature=-1.0)
+    assert w.wedlm_confidence_workspace_bytes(bad) == 0
+    # the fused call never stores logits, so it has nothing to draw from
+    B, W, H = cfg.batch, cfg.window, 64
+    s = w.DecodeStep(c1)
+    i32 = dict(dtype=torch.int32, device="cuda")
+    hs = torch.zeros(B, W, H, dtype=torch.bfloat16, device="cuda")
+    emb = torch.zeros(cfg.vocab, H, dtype=torch.bfloat16, device="cuda")
+    tok = torch.zeros(B, W, **i32)
+    fil = torch.zeros(B, W, dtype=torch.uint8, device="cuda")
+    pl = torch.zeros(B, **i32)
+    s.reorder(fil, tok, pl)
+    ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c1), dtype=torch.uint8, device="cuda")
+    with pytest.raises(w.WedlmError) as ei:
+        w.wedlm_lmhead_confidence_commit(c1, hs, emb, None, 0.0, s.perm, s.n_filled, s.n_commit, tok, fil, pl, None, None,
+                                         s.argmax, s.maxprob, s.entropy, s.lse, s.committed_tokens, s.committed_count,
+                                         s.filled_count, ws)
+    assert ei.value.code == -2
