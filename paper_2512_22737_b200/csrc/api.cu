@@ -138,7 +138,7 @@ const char* wedlm_strerror(int code) {
   }
 }
 
-int wedlm_version(void) { return 100; }
+int wedlm_version(void) { return 200; }
 
 unsigned long long wedlm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
