@@ -629,6 +629,71 @@ def run_lmhead(args):
     return 0
 
 
+# ----------------------------------------------------------------------------------------------
+# Dual-Stream Masking training forward (Section 4.2): attention over the two-stream input
+# ----------------------------------------------------------------------------------------------
+def run_dual_stream(args):
+    import statistics
+    import torch
+    from paper_2512_22737_b200 import build as b
+    from workloads import DS_CONFIGS, make_dual_stream
+    b.build()
+    import paper_2512_22737_b200 as w
+    torch.cuda.set_device(0)
+    out = {}
+    for name in args.ds_configs:
+        c = DS_CONFIGS[name]
+        inp = make_dual_stream(c)
+        cfg = w.make_config(batch=c.n_seq, window=c.block, n_q_heads=c.n_q_heads, n_kv_heads=c.n_kv_heads,
+                            head_dim=c.head_dim, page_size=c.page_size, vocab=c.vocab, dtype=c.dtype,
+                            rope_theta=c.rope_theta, mask_token_id=c.mask_token_id, attn_impl=args.attn)
+        N, K, L, B, Lp = c.n_seq, c.n_blocks, c.seq_len, c.block, c.padded_len
+        i32 = dict(dtype=torch.int32, device="cuda")
+        tokens, masked = w.to_device(inp["tokens"]), w.to_device(inp["masked"])
+        x, pin = torch.empty(N, 2, Lp, **i32), torch.empty(N, 2, Lp, **i32)
+        q, k, v = (w.to_device(inp[t]) for t in ("q", "k", "v"))
+        o = torch.empty_like(q)
+        ws = torch.empty(w.wedlm_dual_stream_workspace_bytes(cfg, K), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, **i32)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")       # larger than L2
+        ts, launches0 = [], w.wedlm_launch_count()
+        for it in range(args.warmup + args.steps):
+            flush.fill_(it & 0xff)
+            a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            w.wedlm_dual_stream_construct(cfg, K, L, tokens, masked, x, pin)
+            w.wedlm_dual_stream_attn(cfg, K, q, k, v, pin, o, ws, status)
+            e.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(e))
+        assert int(status.item()) == 0
+        launches = (w.wedlm_launch_count() - launches0) // (args.warmup + args.steps)
+        ts = ts[args.warmup:]
+        ms = statistics.median(ts)
+        # visible keys per row: k*B + r + 1, both streams; QK^T and PV are 2*D flops per (row, key, head) each
+        keys = 2 * sum((i // B) * B + (i % B) + 1 for i in range(L))
+        flops = 4.0 * c.head_dim * c.n_q_heads * keys * N
+        elem = 2 if c.dtype == "bf16" else 4
+        io_bytes = N * 2 * Lp * (2 * c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim * elem      # q, out, k, v once
+        out[name] = {"ms_median": ms, "ms_min": min(ts), "tokens_per_s": N * L / (ms * 1e-3),
+                     "attention_TFLOPs": flops / (ms * 1e-3) / 1e12, "flops": flops, "io_bytes": io_bytes,
+                     "launches_per_forward": int(launches), "seq_len": L, "block": B, "n_seq": N}
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak, kind = float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        peak, kind = 1590.0, "fallback"
+    first = out[args.ds_configs[0]]
+    line = {"metric": "dual_stream_attention_tokens_per_s", "value": first["tokens_per_s"], "unit": "tokens/s", "n_gpus": 1,
+            "dtype": "bf16", "data": "synthetic", "higher_is_better": True,
+            "config": {"workload": args.ds_configs[0], "l2": "flushed between iterations", "attn_impl": args.attn},
+            "roofline": {"bound": "tensor", "achieved": first["attention_TFLOPs"], "peak": peak, "peak_kind": kind,
+                         "unit": "TFLOP/s", "frac": first["attention_TFLOPs"] / peak, "traffic": None},
+            "results": out}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -643,6 +708,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling runs)")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="Sample() temperature of the step workloads (0 = arg-max, the headline configuration)")
+    ap.add_argument("--ds-configs", type=lambda s: s.split(","), default=["ds_4k", "ds_8k"],
+                    help="dual-stream training-forward shapes timed by --workload dual_stream")
     ap.add_argument("--loop-batch", type=int, default=16)
     ap.add_argument("--loop-new-tokens", type=int, default=1024)
     ap.add_argument("--loop-windows", type=lambda s: [int(x) for x in s.split(",")], default=[16, 2, 1])
@@ -659,6 +726,8 @@ def main():
         return run_loop(args)
     if args.workload == "lmhead":
         return run_lmhead(args)
+    if args.workload == "dual_stream":
+        return run_dual_stream(args)
     args.warmup = max(args.warmup, 3) if args.impl == "product" else args.warmup
     if args.impl == "reference":
         return run_reference(args)

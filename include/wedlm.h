@@ -15,6 +15,7 @@
  *                            selection by distance-adjusted entropy (Eq. 11), then Commit,
  *                            Predict and Refill of Algorithm 1.
  *   wedlm_window_refill      Commit + shift + Refill alone.
+ *   wedlm_dual_stream_*      training side (Section 4.2): two-stream input construction and its attention.
  *
  * Conventions common to every call
  *   - Every pointer named below is a DEVICE pointer unless it is the config or says "host".
@@ -294,6 +295,44 @@ int wedlm_window_refill(const wedlm_config_t* cfg, const int32_t* n_commit,
                         int32_t* window_tokens, uint8_t* filled, int32_t* prefix_len,
                         int32_t* window_len, int32_t* remaining_budget,
                         int32_t* committed_tokens, int32_t* committed_count, void* stream);
+
+/*
+ * Dual-Stream Masking for training (Section 4.2): the forward-pass pieces that need no data or weights.
+ *
+ * cfg fields used: batch = N sequences, window = block size B, n_q_heads, n_kv_heads, head_dim, page_size
+ * (B must be a multiple of it; the tensor-core path needs page_size 16), dtype, rope_style, rope_theta,
+ * softmax_scale, attn_impl, mask_token_id.  Every other field is ignored.
+ * n_blocks = K = ceil(L / B) blocks per stream; Lp = K*B rows per stream (rows at or beyond L are padding).
+ * All pointers are device pointers.
+ *
+ * wedlm_dual_stream_construct - Eq. 8-9 with block-wise masking and intra-block Topological Reordering:
+ *   tokens   in  i32 [N,L]     the clean sequence
+ *   masked   in  u8  [N,L]     non-zero = this logical position of the prediction stream is masked
+ *   x_input  out i32 [N,2,Lp]  stream 0 = memory stream (tokens as they are), stream 1 = prediction stream:
+ *                              inside every block the observed tokens first, the masked ones (mask_token_id)
+ *                              last, both in ascending logical order; padding rows carry mask_token_id
+ *   p_input  out i32 [N,2,Lp]  logical position of every physical row; both streams use positions 0..L-1
+ *   is_mask  out u8  [N,Lp] or NULL   prediction-stream rows that are masked (the rows that enter the loss)
+ *   n_observed out i32 [N,K] or NULL  observed tokens per block
+ *
+ * wedlm_dual_stream_attn - attention under the pattern of the "Attention Pattern" paragraph: a row of block k,
+ * in either stream, sees the memory-stream rows at positions below k*B and the rows of its own block that are
+ * physically not later than itself (for the memory stream this is plain causal attention).  RoPE at p_input.
+ *   q        in  [N,2,Lp,Hq,D]   physical order (stream 0 memory, stream 1 prediction), un-rotated
+ *   k, v     in  [N,2,Lp,Hkv,D]
+ *   out      out [N,2,Lp,Hq,D]   rows of padding slots are computed like any other row and carry no meaning
+ *   workspace    wedlm_dual_stream_workspace_bytes(cfg, n_blocks) bytes, 16-byte aligned: rotated K and V of
+ *                both streams in page layout, one page table per (sequence, stream, block), scratch
+ *   status   in/out i32 [1] or NULL, WEDLM_STATUS_* bits
+ * Padding rows must hold finite numbers.  Returns WEDLM_ERR_UNSUPPORTED if B is not a multiple of page_size.
+ */
+int wedlm_dual_stream_construct(const wedlm_config_t* cfg, int32_t n_blocks, int32_t seq_len,
+                                const int32_t* tokens, const uint8_t* masked, int32_t* x_input,
+                                int32_t* p_input, uint8_t* is_mask, int32_t* n_observed, void* stream);
+size_t wedlm_dual_stream_workspace_bytes(const wedlm_config_t* cfg, int32_t n_blocks);
+int wedlm_dual_stream_attn(const wedlm_config_t* cfg, int32_t n_blocks, const void* q, const void* k,
+                           const void* v, const int32_t* p_input, void* out, void* workspace,
+                           size_t workspace_bytes, int32_t* status, void* stream);
 
 #ifdef __cplusplus
 }

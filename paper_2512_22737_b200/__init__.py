@@ -17,6 +17,9 @@ from .binding import (  # noqa: F401
     wedlm_confidence_commit,
     wedlm_confidence_commit_static,
     wedlm_confidence_workspace_bytes,
+    wedlm_dual_stream_attn,
+    wedlm_dual_stream_construct,
+    wedlm_dual_stream_workspace_bytes,
     wedlm_kv_append,
     wedlm_launch_count,
     wedlm_lmhead_confidence_commit,

@@ -101,6 +101,12 @@ def load_library() -> ctypes.CDLL:
                                                    i32p, vp, ctypes.c_size_t, vp]
     lib.wedlm_window_refill.restype = ctypes.c_int
     lib.wedlm_window_refill.argtypes = [cfgp, i32p, i32p, u8p, i32p, i32p, i32p, i32p, i32p, vp]
+    lib.wedlm_dual_stream_construct.restype = ctypes.c_int
+    lib.wedlm_dual_stream_construct.argtypes = [cfgp, ctypes.c_int32, ctypes.c_int32, i32p, u8p, i32p, i32p, u8p, i32p, vp]
+    lib.wedlm_dual_stream_workspace_bytes.restype = ctypes.c_size_t
+    lib.wedlm_dual_stream_workspace_bytes.argtypes = [cfgp, ctypes.c_int32]
+    lib.wedlm_dual_stream_attn.restype = ctypes.c_int
+    lib.wedlm_dual_stream_attn.argtypes = [cfgp, ctypes.c_int32, vp, vp, vp, i32p, vp, vp, ctypes.c_size_t, i32p, vp]
     _lib = lib
     return lib
 
@@ -289,6 +295,28 @@ def wedlm_window_refill(cfg, n_commit, window_tokens, filled, prefix_len, window
         _ptr(filled, u8, "filled"), _ptr(prefix_len, i32, "prefix_len"), _ptr(window_len, i32, "window_len"),
         _ptr(remaining_budget, i32, "remaining_budget"), _ptr(committed_tokens, i32, "committed_tokens"),
         _ptr(committed_count, i32, "committed_count"), _stream(stream)), "wedlm_window_refill")
+
+
+def wedlm_dual_stream_construct(cfg, n_blocks, seq_len, tokens, masked, x_input, p_input, is_mask=None, n_observed=None,
+                                stream=None) -> None:
+    i32, u8 = torch.int32, torch.uint8
+    _check(load_library().wedlm_dual_stream_construct(
+        ctypes.byref(cfg), ctypes.c_int32(n_blocks), ctypes.c_int32(seq_len), _ptr(tokens, i32, "tokens"),
+        _ptr(masked, u8, "masked"), _ptr(x_input, i32, "x_input"), _ptr(p_input, i32, "p_input"),
+        _ptr(is_mask, u8, "is_mask"), _ptr(n_observed, i32, "n_observed"), _stream(stream)), "wedlm_dual_stream_construct")
+
+
+def wedlm_dual_stream_workspace_bytes(cfg, n_blocks) -> int:
+    return int(load_library().wedlm_dual_stream_workspace_bytes(ctypes.byref(cfg), ctypes.c_int32(n_blocks)))
+
+
+def wedlm_dual_stream_attn(cfg, n_blocks, q, k, v, p_input, out, workspace, status=None, stream=None) -> None:
+    dt = cfg.torch_dtype
+    _check(load_library().wedlm_dual_stream_attn(
+        ctypes.byref(cfg), ctypes.c_int32(n_blocks), _ptr(q, dt, "q"), _ptr(k, dt, "k"), _ptr(v, dt, "v"),
+        _ptr(p_input, torch.int32, "p_input"), _ptr(out, dt, "out"), _ptr(workspace, None, "workspace"),
+        ctypes.c_size_t(workspace.numel() * workspace.element_size()), _ptr(status, torch.int32, "status"),
+        _stream(stream)), "wedlm_dual_stream_attn")
 
 
 # ----------------------------------------------------------------------------------------

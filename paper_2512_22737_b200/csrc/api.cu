@@ -278,6 +278,90 @@ int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, co
                             committed_count, filled_count, st);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Dual-Stream Masking (Section 4.2)
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+struct DualPlan {
+  wedlm_config_t ic;          // the batch of (sequence, stream, block) windows
+  size_t pool_bytes, table_bytes, prefix_bytes, attn_bytes, total_bytes;
+};
+
+int plan_dual_stream(const wedlm_config_t* cfg, int32_t n_blocks, DualPlan* out) {
+  if (cfg == nullptr || n_blocks < 1) return WEDLM_ERR_INVALID_ARG;
+  if (cfg->batch < 0 || cfg->window < 1 || cfg->window > 1024) return WEDLM_ERR_INVALID_ARG;
+  if (cfg->page_size < 1 || cfg->window % cfg->page_size != 0) return WEDLM_ERR_UNSUPPORTED;   // blocks own whole pages
+  const long long units = (long long)cfg->batch * 2 * n_blocks;
+  const long long pages_per_stream = (long long)n_blocks * (cfg->window / cfg->page_size);
+  if (units > 0x7fffffffLL / 4 || units * pages_per_stream > 0x7fffffffLL || (long long)n_blocks * cfg->window > 0x7fffffffLL / 2)
+    return WEDLM_ERR_UNSUPPORTED;
+  DualPlan p{};
+  p.ic = *cfg;
+  p.ic.batch = (int32_t)units;
+  p.ic.max_pages_per_seq = (int32_t)pages_per_stream;
+  p.ic.num_pages = (int32_t)((long long)cfg->batch * 2 * pages_per_stream);
+  p.ic.max_prefix_len = (n_blocks - 1) * cfg->window;
+  p.ic.commit_mode = WEDLM_COMMIT_STREAMING;
+  if (cfg->batch == 0) p.ic.num_pages = 1;
+  int rc = check_config(&p.ic, true, false);
+  if (rc != WEDLM_OK) return rc;
+  const size_t elem = cfg->dtype == WEDLM_DTYPE_BF16 ? 2 : 4;
+  p.pool_bytes = align_up((size_t)units * cfg->window * cfg->n_kv_heads * cfg->head_dim * elem, 256);
+  p.table_bytes = align_up((size_t)units * pages_per_stream * sizeof(int32_t), 256);
+  p.prefix_bytes = align_up((size_t)units * sizeof(int32_t), 256);
+  p.attn_bytes = align_up(plan_attention(&p.ic).total_bytes, 256);
+  p.total_bytes = 2 * p.pool_bytes + p.table_bytes + p.prefix_bytes + p.attn_bytes;
+  *out = p;
+  return WEDLM_OK;
+}
+
+}  // namespace
+
+int wedlm_dual_stream_construct(const wedlm_config_t* cfg, int32_t n_blocks, int32_t seq_len, const int32_t* tokens,
+                                const uint8_t* masked, int32_t* x_input, int32_t* p_input, uint8_t* is_mask,
+                                int32_t* n_observed, void* stream) {
+  if (cfg == nullptr || n_blocks < 1 || cfg->batch < 0 || cfg->window < 1 || cfg->window > 1024) return WEDLM_ERR_INVALID_ARG;
+  if (seq_len < 1 || (long long)seq_len > (long long)n_blocks * cfg->window ||
+      (long long)seq_len <= (long long)(n_blocks - 1) * cfg->window)
+    return WEDLM_ERR_INVALID_ARG;                 // n_blocks must be ceil(seq_len / window)
+  if ((long long)cfg->batch * n_blocks > 0x7fffffffLL) return WEDLM_ERR_UNSUPPORTED;
+  if (cfg->batch == 0) return WEDLM_OK;
+  if (!tokens || !masked || !x_input || !p_input) return WEDLM_ERR_INVALID_ARG;
+  return launch_dual_stream_construct(cfg->batch, seq_len, cfg->window, n_blocks, cfg->mask_token_id, tokens, masked,
+                                      x_input, p_input, is_mask, n_observed, (cudaStream_t)stream);
+}
+
+size_t wedlm_dual_stream_workspace_bytes(const wedlm_config_t* cfg, int32_t n_blocks) {
+  DualPlan p;
+  if (plan_dual_stream(cfg, n_blocks, &p) != WEDLM_OK) return 0;
+  return p.total_bytes ? p.total_bytes : 256;
+}
+
+int wedlm_dual_stream_attn(const wedlm_config_t* cfg, int32_t n_blocks, const void* q, const void* k, const void* v,
+                           const int32_t* p_input, void* out, void* workspace, size_t workspace_bytes, int32_t* status,
+                           void* stream) {
+  DualPlan p;
+  int rc = plan_dual_stream(cfg, n_blocks, &p);
+  if (rc != WEDLM_OK) return rc;
+  if (cfg->batch == 0) return WEDLM_OK;
+  if (!q || !k || !v || !p_input || !out || !workspace) return WEDLM_ERR_INVALID_ARG;
+  if (!aligned16(workspace)) return WEDLM_ERR_INVALID_ARG;
+  if (workspace_bytes < p.total_bytes) return WEDLM_ERR_WORKSPACE_TOO_SMALL;
+  char* ws = static_cast<char*>(workspace);
+  void* k_pool = ws;
+  void* v_pool = ws + p.pool_bytes;
+  int32_t* table = reinterpret_cast<int32_t*>(ws + 2 * p.pool_bytes);
+  int32_t* prefix = reinterpret_cast<int32_t*>(ws + 2 * p.pool_bytes + p.table_bytes);
+  void* attn_ws = ws + 2 * p.pool_bytes + p.table_bytes + p.prefix_bytes;
+  rc = launch_dual_stream_tables(p.ic.batch, n_blocks, cfg->window, cfg->page_size, table, prefix, (cudaStream_t)stream);
+  if (rc != WEDLM_OK) return rc;
+  // every unit rotates its rows at p_input and stages them into its own pages; the attention of unit (n, s, k)
+  // then walks memory pages [0, k*B) and its own block behind them
+  return wedlm_window_attn(&p.ic, q, k, v, k_pool, v_pool, table, prefix, p_input, out, nullptr, attn_ws, p.attn_bytes,
+                           status, stream);
+}
+
 int wedlm_window_refill(const wedlm_config_t* cfg, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
                         int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
                         int32_t* committed_tokens, int32_t* committed_count, void* stream) {

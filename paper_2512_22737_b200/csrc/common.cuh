@@ -96,6 +96,13 @@ int launch_lmhead_conf(const Shape& s, int hidden, const void* hidden_states, co
                        float tilt, const int32_t* n_filled, const int32_t* window_len, void* partials, int* n_tiles_out,
                        cudaStream_t st);
 
+// Dual-Stream Masking (training forward): input construction and the per-unit page tables.
+int launch_dual_stream_construct(int N, int L, int B, int K, int mask_id, const int32_t* tokens, const uint8_t* masked,
+                                 int32_t* x_input, int32_t* p_input, uint8_t* is_mask, int32_t* n_observed,
+                                 cudaStream_t st);
+int launch_dual_stream_tables(int n_units, int K, int B, int page, int32_t* block_table, int32_t* prefix_len,
+                              cudaStream_t st);
+
 int launch_window_refill(const Shape& s, const wedlm_config_t* cfg, const int32_t* n_commit, int32_t* window_tokens,
                          uint8_t* filled, int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
                          int32_t* committed_tokens, int32_t* committed_count, cudaStream_t st);

@@ -1,0 +1,158 @@
+"""GPU-vs-oracle parity of Dual-Stream Masking (Section 4.2): the two-stream input construction (bit-exact)
+and the attention its mask defines (per output vector max|err| / max|ref| <= 1e-2, bf16 in, fp32 accumulate)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2512_22737_b200 as w
+from oracle import dual_stream_oracle as ds
+from workloads import DS_CONFIGS, make_dual_stream
+
+pytestmark = pytest.mark.gpu
+
+ATTN_REL_TOL = 1e-2
+
+
+def _cfg(c, attn_impl="auto"):
+    return w.make_config(batch=c.n_seq, window=c.block, n_q_heads=c.n_q_heads, n_kv_heads=c.n_kv_heads,
+                         head_dim=c.head_dim, page_size=c.page_size, vocab=c.vocab, dtype=c.dtype,
+                         rope_theta=c.rope_theta, mask_token_id=c.mask_token_id, attn_impl=attn_impl)
+
+
+def _construct(c, inp):
+    cfg = _cfg(c)
+    N, K, Lp = c.n_seq, c.n_blocks, c.padded_len
+    i32 = dict(dtype=torch.int32, device="cuda")
+    x = torch.full((N, 2, Lp), -7, **i32)
+    p = torch.full((N, 2, Lp), -7, **i32)
+    im = torch.full((N, Lp), 9, dtype=torch.uint8, device="cuda")
+    nobs = torch.full((N, K), -7, **i32)
+    w.wedlm_dual_stream_construct(cfg, K, c.seq_len, w.to_device(inp["tokens"]), w.to_device(inp["masked"]), x, p, im, nobs)
+    torch.cuda.synchronize()
+    return x, p, im, nobs
+
+
+def _check_construct(c, inp, x, p, im, nobs):
+    L, B, Lp = c.seq_len, c.block, c.padded_len
+    xh, ph, imh, nh = x.cpu().numpy(), p.cpu().numpy(), im.cpu().numpy(), nobs.cpu().numpy()
+    for n in range(c.n_seq):
+        ref = ds.construct(inp["tokens"][n], inp["masked"][n], B, c.mask_token_id)
+        np.testing.assert_array_equal(xh[n, 0, :L], ref["x_input"][:L])
+        np.testing.assert_array_equal(xh[n, 1, :L], ref["x_input"][L:])
+        np.testing.assert_array_equal(ph[n, 0, :L], ref["p_input"][:L])
+        np.testing.assert_array_equal(ph[n, 1, :L], ref["p_input"][L:])
+        np.testing.assert_array_equal(imh[n, :L], ref["is_mask"].astype(np.uint8))
+        # padding rows: mask id, own index as position, not part of the loss
+        assert (xh[n, :, L:] == c.mask_token_id).all() and (imh[n, L:] == 0).all()
+        np.testing.assert_array_equal(ph[n, 0, L:], np.arange(L, Lp))
+        np.testing.assert_array_equal(ph[n, 1, L:], np.arange(L, Lp))
+        for kb in range(c.n_blocks):
+            blk = inp["masked"][n, kb * B:min((kb + 1) * B, L)]
+            assert nh[n, kb] == int((blk == 0).sum())
+
+
+def _attend(c, inp, p_input, attn_impl):
+    cfg = _cfg(c, attn_impl)
+    K = c.n_blocks
+    q, k, v = (w.to_device(inp[name]) for name in ("q", "k", "v"))
+    out = torch.zeros_like(q)
+    ws = torch.empty(w.wedlm_dual_stream_workspace_bytes(cfg, K), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    w.wedlm_dual_stream_attn(cfg, K, q, k, v, p_input, out, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return out.to(torch.float64).cpu().numpy()
+
+
+def _oracle_inputs(c, inp, n, p_input_host):
+    L = c.seq_len
+    cat = lambda a: np.concatenate([a[n, 0, :L], a[n, 1, :L]], axis=0)
+    return cat(inp["q"]), cat(inp["k"]), cat(inp["v"]), np.concatenate([p_input_host[n, 0, :L], p_input_host[n, 1, :L]])
+
+
+def _vec_err(got, ref):
+    return np.abs(got - ref).max(axis=-1) / np.maximum(np.abs(ref).max(axis=-1), 1e-30)
+
+
+@pytest.mark.parametrize("name,kw", [("ds_small", {}), ("ds_small", dict(seq_len=128, block=16)), ("ds_small", dict(seq_len=1)),
+                                     ("ds_small", dict(seq_len=97, block=64, n_seq=3)), ("ds_small", dict(seq_len=40, block=8, page_size=8))])
+def test_construction_is_bit_exact(name, kw):
+    c = DS_CONFIGS[name].replace(**kw)
+    inp = make_dual_stream(c, seed=17)
+    _check_construct(c, inp, *_construct(c, inp))
+
+
+@pytest.mark.parametrize("impl", ["tensor", "generic"])
+@pytest.mark.parametrize("kw", [{}, dict(seq_len=128, block=16), dict(seq_len=70, block=64, n_q_heads=8, n_kv_heads=8)])
+def test_small_sequences_every_row(impl, kw):
+    c = DS_CONFIGS["ds_small"].replace(**kw)
+    inp = make_dual_stream(c, seed=23)
+    x, p, im, nobs = _construct(c, inp)
+    got = _attend(c, inp, p, impl)
+    ph = p.cpu().numpy()
+    L = c.seq_len
+    worst = 0.0
+    for n in range(c.n_seq):
+        q, k, v, pos = _oracle_inputs(c, inp, n, ph)
+        ref = ds.attention(q, k, v, pos, c.block, theta=c.rope_theta)
+        err = np.concatenate([_vec_err(got[n, 0, :L], ref[:L]), _vec_err(got[n, 1, :L], ref[L:])])
+        assert np.isfinite(got[n]).all()
+        assert err.max() <= ATTN_REL_TOL, err.max()
+        worst = max(worst, float(err.max()))
+    print("dual-stream attention error", worst)
+
+
+def test_fp32_generic_path_small_heads():
+    c = DS_CONFIGS["ds_small"].replace(seq_len=45, block=8, page_size=8, n_q_heads=4, n_kv_heads=2, head_dim=64, dtype="f32",
+                                       vocab=1001, rope_theta=1.0e4)
+    inp = make_dual_stream(c, seed=29)
+    x, p, im, nobs = _construct(c, inp)
+    got = _attend(c, inp, p, "auto")
+    ph = p.cpu().numpy()
+    L = c.seq_len
+    for n in range(c.n_seq):
+        q, k, v, pos = _oracle_inputs(c, inp, n, ph)
+        ref = ds.attention(q, k, v, pos, c.block, theta=c.rope_theta)
+        err = np.concatenate([_vec_err(got[n, 0, :L], ref[:L]), _vec_err(got[n, 1, :L], ref[L:])])
+        assert err.max() <= 1e-4
+
+
+def test_4k_context_sampled_rows_and_clean_copy_invariant():
+    c = DS_CONFIGS["ds_4k"]
+    inp = make_dual_stream(c, seed=31)
+    x, p, im, nobs = _construct(c, inp)
+    _check_construct(c, inp, x, p, im, nobs)
+    got = _attend(c, inp, p, "auto")
+    ph = p.cpu().numpy()
+    L = c.seq_len
+    q, k, v, pos = _oracle_inputs(c, inp, 0, ph)
+    g = np.random.default_rng(5)
+    rows = sorted(set(g.integers(0, 2 * L, size=20).tolist()) | {0, L - 1, L, L + 31, L + 32, 2 * L - 1})
+    ref = ds.attention(q, k, v, pos, c.block, theta=c.rope_theta, rows=rows)
+    for a in rows:
+        s, i = divmod(a, L)
+        err = _vec_err(got[0, s, i], ref[a])
+        assert err.max() <= ATTN_REL_TOL, (a, err.max())
+    # nothing masked and the prediction stream a copy of the memory stream: both streams must agree row for row
+    inp2 = dict(inp)
+    inp2["masked"] = np.zeros_like(inp["masked"])
+    for name in ("q", "k", "v"):
+        t = inp[name].copy()
+        t[:, 1] = t[:, 0]
+        inp2[name] = t
+    x2, p2, _, _ = _construct(c, inp2)
+    assert torch.equal(p2[:, 0], p2[:, 1])
+    got2 = _attend(c, inp2, p2, "auto")
+    err = _vec_err(got2[0, 1, :L], got2[0, 0, :L])
+    assert err.max() <= 2e-2, err.max()           # two bf16 computations of the same quantity
+
+
+def test_blocks_must_own_whole_pages():
+    c = DS_CONFIGS["ds_small"].replace(block=4)
+    cfg = _cfg(c)
+    assert w.wedlm_dual_stream_workspace_bytes(cfg, c.n_blocks) == 0
+    t = torch.zeros(16, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(w.WedlmError) as ei:
+        w.wedlm_dual_stream_attn(cfg, c.n_blocks, t, t, t, torch.zeros(4, dtype=torch.int32, device="cuda"), t,
+                                 torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert ei.value.code == -2

@@ -24,3 +24,4 @@ from .synth import (  # noqa: F401
     bf16_to_f32,
     BASE_SEED,
 )
+from .dual_stream import DualStreamConfig, DS_CONFIGS, make_dual_stream  # noqa: F401,E402
