@@ -15,6 +15,7 @@
  *                            selection by distance-adjusted entropy (Eq. 11), then Commit,
  *                            Predict and Refill of Algorithm 1.
  *   wedlm_window_refill      Commit + shift + Refill alone.
+ *   wedlm_step_host          the three calls above for step inputs that live in host memory.
  *   wedlm_dual_stream_*      training side (Section 4.2): two-stream input construction and its attention.
  *
  * Conventions common to every call
@@ -295,6 +296,34 @@ int wedlm_window_refill(const wedlm_config_t* cfg, const int32_t* n_commit,
                         int32_t* window_tokens, uint8_t* filled, int32_t* prefix_len,
                         int32_t* window_len, int32_t* remaining_budget,
                         int32_t* committed_tokens, int32_t* committed_count, void* stream);
+
+/*
+ * One whole step of Algorithm 1 (reorder -> window attention -> confidence / commit / refill) for callers whose
+ * step inputs live in HOST memory.  The call enqueues, on `stream`: the host-to-device copies of the inputs into
+ * `workspace`, the kernels of wedlm_reorder, wedlm_window_attn and wedlm_confidence_commit, and the device-to-host
+ * copies of the results; it returns without waiting (synchronise the stream before reading the outputs).  Use
+ * page-locked host memory, or the copies serialise with the host.
+ *   h_filled, h_window_tokens, h_prefix_len   host, in/out: the window state, updated in place by the step
+ *   h_window_len, h_remaining_budget          host, in/out, each may be NULL (meaning as in wedlm_confidence_commit)
+ *   h_block_table, h_q, h_k, h_v, h_logits    host, in: layouts as in wedlm_window_attn / wedlm_confidence_commit.
+ *       Of the logits only the rows the step reads are sent: after reordering these are, per sequence, the physical
+ *       rows [n_filled, window_len).  The CPU reads h_filled (and h_window_len) DURING this call to find them, so
+ *       both must be final when it is made.
+ *   k_cache, v_cache                          device, resident cache pool (the window's K/V are staged into it)
+ *   h_committed_tokens [B,W], h_committed_count [B], h_filled_count [B] (may be NULL)   host, out
+ *   workspace       device, wedlm_step_host_workspace_bytes(cfg) bytes, 16-byte aligned; holds the device copies of
+ *                   every input, every intermediate and output of the three calls, and their scratch
+ *   attn_out        host pointer to a device pointer, or NULL: receives the address (inside workspace) of the
+ *                   attention output [B,W,Hq,D] for the layers that follow
+ *   status          device i32 [1] or NULL
+ */
+size_t wedlm_step_host_workspace_bytes(const wedlm_config_t* cfg);
+int wedlm_step_host(const wedlm_config_t* cfg, uint8_t* h_filled, int32_t* h_window_tokens, int32_t* h_prefix_len,
+                    int32_t* h_window_len, int32_t* h_remaining_budget, const int32_t* h_block_table,
+                    const void* h_q, const void* h_k, const void* h_v, const void* h_logits,
+                    void* k_cache, void* v_cache, int32_t* h_committed_tokens, int32_t* h_committed_count,
+                    int32_t* h_filled_count, void* workspace, size_t workspace_bytes, void** attn_out,
+                    int32_t* status, void* stream);
 
 /*
  * Dual-Stream Masking for training (Section 4.2): the forward-pass pieces that need no data or weights.

@@ -27,6 +27,8 @@ from .binding import (  # noqa: F401
     wedlm_profile_next_attn,
     wedlm_reorder,
     wedlm_selftest_wait_expiry,
+    wedlm_step_host,
+    wedlm_step_host_workspace_bytes,
     wedlm_strerror,
     wedlm_version,
     wedlm_window_attn,

@@ -101,6 +101,10 @@ def load_library() -> ctypes.CDLL:
                                                    i32p, vp, ctypes.c_size_t, vp]
     lib.wedlm_window_refill.restype = ctypes.c_int
     lib.wedlm_window_refill.argtypes = [cfgp, i32p, i32p, u8p, i32p, i32p, i32p, i32p, i32p, vp]
+    lib.wedlm_step_host_workspace_bytes.restype = ctypes.c_size_t
+    lib.wedlm_step_host_workspace_bytes.argtypes = [cfgp]
+    lib.wedlm_step_host.restype = ctypes.c_int
+    lib.wedlm_step_host.argtypes = [cfgp] + [vp] * 15 + [vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_void_p), i32p, vp]
     lib.wedlm_dual_stream_construct.restype = ctypes.c_int
     lib.wedlm_dual_stream_construct.argtypes = [cfgp, ctypes.c_int32, ctypes.c_int32, i32p, u8p, i32p, i32p, u8p, i32p, vp]
     lib.wedlm_dual_stream_workspace_bytes.restype = ctypes.c_size_t
@@ -295,6 +299,43 @@ def wedlm_window_refill(cfg, n_commit, window_tokens, filled, prefix_len, window
         _ptr(filled, u8, "filled"), _ptr(prefix_len, i32, "prefix_len"), _ptr(window_len, i32, "window_len"),
         _ptr(remaining_budget, i32, "remaining_budget"), _ptr(committed_tokens, i32, "committed_tokens"),
         _ptr(committed_count, i32, "committed_count"), _stream(stream)), "wedlm_window_refill")
+
+
+def _hptr(t: Optional[torch.Tensor], dtype: Optional[torch.dtype], name: str):
+    """Host tensor -> raw pointer (page-locked memory is the caller's business)."""
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor) or t.is_cuda:
+        raise TypeError(f"{name} must be a CPU tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def wedlm_step_host_workspace_bytes(cfg) -> int:
+    return int(load_library().wedlm_step_host_workspace_bytes(ctypes.byref(cfg)))
+
+
+def wedlm_step_host(cfg, h_filled, h_window_tokens, h_prefix_len, h_window_len, h_remaining_budget, h_block_table,
+                    h_q, h_k, h_v, h_logits, k_cache, v_cache, h_committed_tokens, h_committed_count, h_filled_count,
+                    workspace, status=None, stream=None) -> int:
+    """One whole step from host tensors (bf16 tensors may be passed as int16/uint16 bit patterns).  Asynchronous
+    on the stream.  Returns the device address of the attention output inside the workspace."""
+    i32, u8 = torch.int32, torch.uint8
+    out_ptr = ctypes.c_void_p()
+    _check(load_library().wedlm_step_host(
+        ctypes.byref(cfg), _hptr(h_filled, u8, "h_filled"), _hptr(h_window_tokens, i32, "h_window_tokens"),
+        _hptr(h_prefix_len, i32, "h_prefix_len"), _hptr(h_window_len, i32, "h_window_len"),
+        _hptr(h_remaining_budget, i32, "h_remaining_budget"), _hptr(h_block_table, i32, "h_block_table"),
+        _hptr(h_q, None, "h_q"), _hptr(h_k, None, "h_k"), _hptr(h_v, None, "h_v"), _hptr(h_logits, None, "h_logits"),
+        _ptr(k_cache, cfg.torch_dtype, "k_cache"), _ptr(v_cache, cfg.torch_dtype, "v_cache"),
+        _hptr(h_committed_tokens, i32, "h_committed_tokens"), _hptr(h_committed_count, i32, "h_committed_count"),
+        _hptr(h_filled_count, i32, "h_filled_count"), _ptr(workspace, None, "workspace"),
+        ctypes.c_size_t(workspace.numel() * workspace.element_size()), ctypes.byref(out_ptr),
+        _ptr(status, i32, "status"), _stream(stream)), "wedlm_step_host")
+    return int(out_ptr.value or 0)
 
 
 def wedlm_dual_stream_construct(cfg, n_blocks, seq_len, tokens, masked, x_input, p_input, is_mask=None, n_observed=None,

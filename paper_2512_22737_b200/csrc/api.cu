@@ -362,6 +362,146 @@ int wedlm_dual_stream_attn(const wedlm_config_t* cfg, int32_t n_blocks, const vo
                            status, stream);
 }
 
+// ---------------------------------------------------------------------------------------------
+// One whole step from host buffers
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+struct HostStepPlan {
+  size_t off_filled, off_tokens, off_prefix, off_wlen, off_budget, off_table, off_q, off_k, off_v, off_logits;
+  size_t off_perm, off_inv, off_pos, off_tokphys, off_nfilled, off_ncommit, off_out, off_argmax, off_maxprob, off_entropy,
+      off_lse, off_ctok, off_ccount, off_fcount, off_attn_ws, off_conf_ws;
+  size_t attn_ws_bytes, conf_ws_bytes, total;
+};
+
+int plan_host_step(const wedlm_config_t* cfg, HostStepPlan* out) {
+  int rc = check_config(cfg, true, true);
+  if (rc != WEDLM_OK) return rc;
+  const size_t B = cfg->batch, W = cfg->window, elem = cfg->dtype == WEDLM_DTYPE_BF16 ? 2 : 4;
+  HostStepPlan p{};
+  size_t at = 0;
+  auto take = [&](size_t bytes) { size_t o = at; at += align_up(bytes ? bytes : 1, 256); return o; };
+  p.off_filled = take(B * W);
+  p.off_tokens = take(B * W * 4);
+  p.off_prefix = take(B * 4);
+  p.off_wlen = take(B * 4);
+  p.off_budget = take(B * 4);
+  p.off_table = take(B * (size_t)cfg->max_pages_per_seq * 4);
+  p.off_q = take(B * W * cfg->n_q_heads * cfg->head_dim * elem);
+  p.off_k = take(B * W * cfg->n_kv_heads * cfg->head_dim * elem);
+  p.off_v = take(B * W * cfg->n_kv_heads * cfg->head_dim * elem);
+  p.off_logits = take(B * W * (size_t)cfg->vocab * elem);
+  p.off_perm = take(B * W * 4);
+  p.off_inv = take(B * W * 4);
+  p.off_pos = take(B * W * 4);
+  p.off_tokphys = take(B * W * 4);
+  p.off_nfilled = take(B * 4);
+  p.off_ncommit = take(B * 4);
+  p.off_out = take(B * W * cfg->n_q_heads * cfg->head_dim * elem);
+  p.off_argmax = take(B * W * 4);
+  p.off_maxprob = take(B * W * 4);
+  p.off_entropy = take(B * W * 4);
+  p.off_lse = take(B * W * 4);
+  p.off_ctok = take(B * W * 4);
+  p.off_ccount = take(B * 4);
+  p.off_fcount = take(B * 4);
+  p.attn_ws_bytes = plan_attention(cfg).total_bytes;
+  p.conf_ws_bytes = confidence_workspace_bytes(cfg);
+  p.off_attn_ws = take(p.attn_ws_bytes);
+  p.off_conf_ws = take(p.conf_ws_bytes);
+  p.total = at;
+  *out = p;
+  return WEDLM_OK;
+}
+
+}  // namespace
+
+size_t wedlm_step_host_workspace_bytes(const wedlm_config_t* cfg) {
+  HostStepPlan p;
+  if (plan_host_step(cfg, &p) != WEDLM_OK) return 0;
+  return p.total;
+}
+
+int wedlm_step_host(const wedlm_config_t* cfg, uint8_t* h_filled, int32_t* h_window_tokens, int32_t* h_prefix_len,
+                    int32_t* h_window_len, int32_t* h_remaining_budget, const int32_t* h_block_table, const void* h_q,
+                    const void* h_k, const void* h_v, const void* h_logits, void* k_cache, void* v_cache,
+                    int32_t* h_committed_tokens, int32_t* h_committed_count, int32_t* h_filled_count, void* workspace,
+                    size_t workspace_bytes, void** attn_out, int32_t* status, void* stream) {
+  HostStepPlan p;
+  int rc = plan_host_step(cfg, &p);
+  if (rc != WEDLM_OK) return rc;
+  if (attn_out) *attn_out = nullptr;
+  if (cfg->batch == 0) return WEDLM_OK;
+  if (!h_filled || !h_window_tokens || !h_prefix_len || !h_block_table || !h_q || !h_k || !h_v || !h_logits || !k_cache ||
+      !v_cache || !h_committed_tokens || !h_committed_count || !workspace)
+    return WEDLM_ERR_INVALID_ARG;
+  if (!aligned16(workspace) || !aligned16(k_cache) || !aligned16(v_cache)) return WEDLM_ERR_INVALID_ARG;
+  if (workspace_bytes < p.total) return WEDLM_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = static_cast<char*>(workspace);
+  const size_t B = cfg->batch, W = cfg->window, elem = cfg->dtype == WEDLM_DTYPE_BF16 ? 2 : 4;
+  auto up = [&](size_t off, const void* src, size_t bytes) {
+    return cudaMemcpyAsync(ws + off, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  };
+  auto down = [&](void* dst, size_t off, size_t bytes) {
+    return cudaMemcpyAsync(dst, ws + off, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  };
+  bool ok = up(p.off_filled, h_filled, B * W) && up(p.off_tokens, h_window_tokens, B * W * 4) &&
+            up(p.off_prefix, h_prefix_len, B * 4) && up(p.off_table, h_block_table, B * (size_t)cfg->max_pages_per_seq * 4) &&
+            up(p.off_q, h_q, B * W * cfg->n_q_heads * cfg->head_dim * elem) &&
+            up(p.off_k, h_k, B * W * cfg->n_kv_heads * cfg->head_dim * elem) &&
+            up(p.off_v, h_v, B * W * cfg->n_kv_heads * cfg->head_dim * elem);
+  if (ok && h_window_len) ok = up(p.off_wlen, h_window_len, B * 4);
+  if (ok && h_remaining_budget) ok = up(p.off_budget, h_remaining_budget, B * 4);
+  if (!ok) return WEDLM_ERR_CUDA;
+  uint8_t* d_filled = reinterpret_cast<uint8_t*>(ws + p.off_filled);
+  int32_t* d_tokens = reinterpret_cast<int32_t*>(ws + p.off_tokens);
+  int32_t* d_prefix = reinterpret_cast<int32_t*>(ws + p.off_prefix);
+  int32_t* d_wlen = h_window_len ? reinterpret_cast<int32_t*>(ws + p.off_wlen) : nullptr;
+  int32_t* d_budget = h_remaining_budget ? reinterpret_cast<int32_t*>(ws + p.off_budget) : nullptr;
+  int32_t* d_perm = reinterpret_cast<int32_t*>(ws + p.off_perm);
+  int32_t* d_pos = reinterpret_cast<int32_t*>(ws + p.off_pos);
+  int32_t* d_nfilled = reinterpret_cast<int32_t*>(ws + p.off_nfilled);
+  int32_t* d_ncommit = reinterpret_cast<int32_t*>(ws + p.off_ncommit);
+  // reorder and attention need only the small inputs; the logits follow
+  rc = wedlm_reorder(cfg, d_filled, d_tokens, d_prefix, d_wlen, d_perm, reinterpret_cast<int32_t*>(ws + p.off_inv), d_pos,
+                     reinterpret_cast<int32_t*>(ws + p.off_tokphys), d_nfilled, d_ncommit, stream);
+  if (rc != WEDLM_OK) return rc;
+  rc = wedlm_window_attn(cfg, ws + p.off_q, ws + p.off_k, ws + p.off_v, k_cache, v_cache,
+                         reinterpret_cast<int32_t*>(ws + p.off_table), d_prefix, d_pos, ws + p.off_out, nullptr,
+                         ws + p.off_attn_ws, p.attn_ws_bytes, status, stream);
+  if (rc != WEDLM_OK) return rc;
+  // Logits: only the rows the confidence pass reads.  After reordering the mask rows of a sequence are the
+  // physical rows [n_filled, window_len), one contiguous range, and n_filled is a count over the host's flags.
+  for (size_t b = 0; b < B; ++b) {
+    long long L = h_window_len ? h_window_len[b] : (long long)W;
+    L = L < 0 ? 0 : (L > (long long)W ? (long long)W : L);
+    long long nf = 0;
+    for (long long j = 0; j < L; ++j) nf += h_filled[b * W + j] != 0;
+    if (L > nf) {
+      const size_t off = (b * W + (size_t)nf) * (size_t)cfg->vocab * elem;
+      if (!up(p.off_logits + off, static_cast<const char*>(h_logits) + off, (size_t)(L - nf) * cfg->vocab * elem))
+        return WEDLM_ERR_CUDA;
+    }
+  }
+  rc = wedlm_confidence_commit(cfg, ws + p.off_logits, d_perm, d_nfilled, d_ncommit, d_tokens, d_filled, d_prefix, d_wlen,
+                               d_budget, reinterpret_cast<int32_t*>(ws + p.off_argmax),
+                               reinterpret_cast<float*>(ws + p.off_maxprob), reinterpret_cast<float*>(ws + p.off_entropy),
+                               reinterpret_cast<float*>(ws + p.off_lse), reinterpret_cast<int32_t*>(ws + p.off_ctok),
+                               reinterpret_cast<int32_t*>(ws + p.off_ccount), reinterpret_cast<int32_t*>(ws + p.off_fcount),
+                               ws + p.off_conf_ws, p.conf_ws_bytes, stream);
+  if (rc != WEDLM_OK) return rc;
+  ok = down(h_committed_tokens, p.off_ctok, B * W * 4) && down(h_committed_count, p.off_ccount, B * 4) &&
+       down(h_filled, p.off_filled, B * W) && down(h_window_tokens, p.off_tokens, B * W * 4) &&
+       down(h_prefix_len, p.off_prefix, B * 4);
+  if (ok && h_filled_count) ok = down(h_filled_count, p.off_fcount, B * 4);
+  if (ok && h_window_len) ok = down(h_window_len, p.off_wlen, B * 4);
+  if (ok && h_remaining_budget) ok = down(h_remaining_budget, p.off_budget, B * 4);
+  if (!ok) return WEDLM_ERR_CUDA;
+  if (attn_out) *attn_out = ws + p.off_out;
+  return WEDLM_OK;
+}
+
 int wedlm_window_refill(const wedlm_config_t* cfg, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
                         int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
                         int32_t* committed_tokens, int32_t* committed_count, void* stream) {

@@ -328,13 +328,20 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
     m = fm[0];
 #pragma unroll
     for (int q = 1; q < kStreamThreads / 32; ++q) m = fmaxf(m, fm[q]);
-    if (m_thread == m) {                             // lowest index attaining the maximum (descending scan)
+    if (m_thread == m) {                             // lowest index attaining the maximum
+      // mx[q] is the maximum over the words i with (i & 3) == q: only those quarters that hold m are searched
       int a = 0x7fffffff;
 #pragma unroll
-      for (int i = kStreamVecs * 4 - 1; i >= 0; --i) {
-        const int e0 = base + ((i >> 2) * kStreamThreads + tid) * 8 + (i & 3) * 2;
-        if (__uint_as_float(w[i] & 0xffff0000u) == m) a = e0 + 1;
-        if (__uint_as_float(w[i] << 16) == m) a = e0;
+      for (int q = 0; q < 4; ++q) {
+        if (__uint_as_float(mx[q] << 16) == m || __uint_as_float(mx[q] & 0xffff0000u) == m) {
+#pragma unroll
+          for (int k = kStreamVecs - 1; k >= 0; --k) {
+            const int i = 4 * k + q;
+            const int e0 = base + (k * kStreamThreads + tid) * 8 + q * 2;
+            if (__uint_as_float(w[i] & 0xffff0000u) == m) a = min(a, e0 + 1);
+            if (__uint_as_float(w[i] << 16) == m) a = min(a, e0);
+          }
+        }
       }
       atomicMin(&fa, a);
     }
