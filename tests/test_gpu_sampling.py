@@ -103,6 +103,16 @@ def test_bf16_full_vocabulary_rows(T):
         assert ng > 0
 
 
+def test_cfg3_batched_serving_full_size_at_the_paper_temperature():
+    """The benchmark's workload and launch configuration (64 windows of 32 slots, V = 151936) at T = 0.1."""
+    cfg = get_config("cfg3_batched")
+    inp = make_step(cfg)
+    step, d, ref = _run(cfg, inp, 0.1, 20251222)
+    c, e, ng = _compare(cfg, inp, step, d, ref)
+    print("cfg3 sampled rows compared", c, "excluded", e, "draws that are not the arg-max", ng)
+    assert c >= cfg.batch // 2 and e <= 2
+
+
 def test_threshold_selection_with_boosts_and_paper_temperature():
     cfg = get_config("cfg2_qwen_b1").replace(vocab=20000, batch=6, boost=14.0, boost_prob=0.6, name="mixed")
     seen = 0
