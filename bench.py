@@ -460,7 +460,10 @@ def run_product(args):
         sampler.stop()
     if rank == 0 and world == 1 and not args.no_cpu:
         cores = len(os.sched_getaffinity(0))
-        n_s = min(wl.cfg.batch, 8 if wl.cfg.batch >= 8 else wl.cfg.batch)
+        # bounded sample: as many sequences of the batch as fit in about 20 s of oracle time
+        n_probe = min(wl.cfg.batch, 4)
+        dt_probe, _ = oracle_step_time(wl.cfg, wl.inp, n_probe)
+        n_s = int(max(n_probe, min(wl.cfg.batch, 20.0 / max(dt_probe / n_probe, 1e-3))))
         log(f"timing the oracle on {n_s} sequences ...")
         dt, c = oracle_step_time(wl.cfg, wl.inp, n_s)
         cpu = {"value": c / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
