@@ -173,3 +173,28 @@ def test_fused_lm_head_refuses_sampling_and_workspace_grows():
                                          s.argmax, s.maxprob, s.entropy, s.lse, s.committed_tokens, s.committed_count,
                                          s.filled_count, ws)
     assert ei.value.code == -2
+
+
+def test_sampled_step_replays_from_a_cuda_graph():
+    """The sampling pass adds a memset node and one kernel whose work list lives on the device: a captured step
+    replayed on restored inputs draws the same tokens as the eager call."""
+    cfg = get_config("cfg2_qwen_b1").replace(vocab=8192, batch=3, prefix_lo=100, prefix_hi=900, tau=50.0, name="graph")
+    inp = make_step(cfg, seed=123)
+    d = {k: w.to_device(v) for k, v in inp.items() if k != "targets"}
+    c = w.config_for(cfg, max_pages_per_seq=inp["block_table"].shape[1], num_pages=inp["k_cache"].shape[0],
+                     max_prefix_len=int(inp["prefix_len"].max()), sample_temperature=1.3, sample_seed=42)
+    step = w.DecodeStep(c)
+    state0 = {k: d[k].clone() for k in ("filled", "window_tokens", "prefix_len")}
+    step.run(d)
+    torch.cuda.synchronize()
+    eager_tokens, eager_argmax = d["window_tokens"].clone(), step.argmax.clone()
+    for k, v in state0.items():
+        d[k].copy_(v)
+    graph = step.capture_graph(d)
+    for _ in range(2):
+        for k, v in state0.items():
+            d[k].copy_(v)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(d["window_tokens"], eager_tokens)
+        assert torch.equal(step.argmax, eager_argmax)
