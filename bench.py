@@ -563,12 +563,13 @@ def run_loop(args):
             dec.tilt = tilt if tilt_name == "literal" else lse0 + tilt
             torch.cuda.synchronize()
             t0 = time.perf_counter()
-            out = dec.generate(N)
+            out = dec.generate(N, use_graph=not args.loop_eager)
             torch.cuda.synchronize()
             dt = time.perf_counter() - t0
             n_gen = sum(len(y) for y in out["y"])
             on_target = sum(int(out["y"][bb] == pt["target"][bb, P:P + N].tolist()) for bb in range(B))
             results.append({"window": W, "commit": mode, "lm_head": "fused" if fused else "gemm+logits",
+                            "replay": "eager" if args.loop_eager else "cuda_graph",
                             "tilt": f"{tilt_name}+{tilt:g}", "tokens_per_s": n_gen / dt, "seconds": dt,
                             "steps": out["steps"], "tokens_per_step_per_seq": n_gen / B / max(out["steps"], 1),
                             "p_cache": out["p_cache"], "sequences_equal_to_target": on_target})
@@ -579,7 +580,7 @@ def run_loop(args):
             "config": {"workload": "cfg5_loop", "batch": B, "prompt": P, "new_tokens": N, "layers": m.n_layers,
                        "tau": args.loop_tau, "lambda": args.loop_lambda,
                        "hidden": H, "lse_of_untilted_logits": lse0,
-                       "timing": "host wall clock around generate(), includes the per-step read-back of commits"},
+                       "timing": "host wall clock around generate(), includes the graph capture and the per-step read-back of commits"},
             "results": results}
     print(json.dumps(line), flush=True)
     return 0
@@ -724,6 +725,8 @@ def main():
     ap.add_argument("--loop-windows", type=lambda s: [int(x) for x in s.split(",")], default=[16, 2, 1])
     ap.add_argument("--loop-fused-windows", type=lambda s: [int(x) for x in s.split(",") if x], default=[],
                     help="windows also run with the LM head fused into the confidence call")
+    ap.add_argument("--loop-eager", action="store_true",
+                    help="launch every step kernel by kernel instead of replaying one captured CUDA graph")
     ap.add_argument("--loop-tau", type=float, default=0.3)
     ap.add_argument("--loop-lambda", type=float, default=0.1)
     ap.add_argument("--loop-block-windows", type=lambda s: [int(x) for x in s.split(",") if x], default=[16],

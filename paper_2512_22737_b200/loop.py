@@ -72,9 +72,15 @@ class StreamingDecoder:
 
     # ------------------------------------------------------------------ dense parts (library GEMMs)
     def _rms(self, x: torch.Tensor, gain: torch.Tensor) -> torch.Tensor:
-        xf = x.float()
-        y = xf * torch.rsqrt(xf.pow(2).mean(-1, keepdim=True) + self.m.rms_eps)
-        return (y * gain.float()).to(self.dtype)
+        return torch.nn.functional.rms_norm(x, (x.shape[-1],), gain, self.m.rms_eps)     # one library kernel
+
+    def _fused(self, l: int):
+        """[wq | wk | wv] and [wg | wu] of layer l as single matrices, so that each pair of projections is one GEMM."""
+        key = f"l{l}.wqkv"
+        if key not in self.wt:
+            self.wt[key] = torch.cat([self.wt[f"l{l}.wq"], self.wt[f"l{l}.wk"], self.wt[f"l{l}.wv"]], dim=1).contiguous()
+            self.wt[f"l{l}.wgu"] = torch.cat([self.wt[f"l{l}.wg"], self.wt[f"l{l}.wu"]], dim=1).contiguous()
+        return self.wt[key], self.wt[f"l{l}.wgu"]
 
     def forward(self, capture_layer: Optional[int] = None, want_logits: bool = True):
         """Causal forward of the reordered window on top of the cache -> logits [B, W, V] (or, with
@@ -85,10 +91,13 @@ class StreamingDecoder:
         h = self.wt["embed"][s.tokens_phys.long()]                       # [B, W, H]
         cap = None
         for l in range(m.n_layers):
+            wqkv, wgu = self._fused(l)
             a = self._rms(h, self.wt[f"l{l}.norm1"])
-            q = (a @ self.wt[f"l{l}.wq"]).view(B, W, m.n_q_heads, m.head_dim).contiguous()
-            k = (a @ self.wt[f"l{l}.wk"]).view(B, W, m.n_kv_heads, m.head_dim).contiguous()
-            v = (a @ self.wt[f"l{l}.wv"]).view(B, W, m.n_kv_heads, m.head_dim).contiguous()
+            nq, nkv = m.n_q_heads * m.head_dim, m.n_kv_heads * m.head_dim
+            qkv = a @ wqkv
+            q = qkv[..., :nq].reshape(B, W, m.n_q_heads, m.head_dim).contiguous()
+            k = qkv[..., nq:nq + nkv].reshape(B, W, m.n_kv_heads, m.head_dim).contiguous()
+            v = qkv[..., nq + nkv:].reshape(B, W, m.n_kv_heads, m.head_dim).contiguous()
             if capture_layer == l:
                 cap = dict(q=q.clone(), k=k.clone(), v=v.clone(), k_cache=self.k_cache[l].clone(),
                            v_cache=self.v_cache[l].clone())
@@ -98,7 +107,8 @@ class StreamingDecoder:
                 cap["kv_slot_idx"] = s.kv_slot_idx.clone()
             h = h + s.out.view(B, W, -1) @ self.wt[f"l{l}.wo"]
             mm = self._rms(h, self.wt[f"l{l}.norm2"])
-            h = h + (torch.nn.functional.silu(mm @ self.wt[f"l{l}.wg"]) * (mm @ self.wt[f"l{l}.wu"])) @ self.wt[f"l{l}.wd"]
+            gu = mm @ wgu
+            h = h + (torch.nn.functional.silu(gu[..., :m.ffn]) * gu[..., m.ffn:]) @ self.wt[f"l{l}.wd"]
         hn = self._rms(h, self.wt["norm_f"])
         if not want_logits:
             return hn.contiguous(), cap
@@ -172,9 +182,33 @@ class StreamingDecoder:
             return s.committed_count, s.committed_tokens, cap
         return s.committed_count, s.committed_tokens
 
-    def generate(self, max_new_tokens: int, max_steps: int = 1_000_000) -> Dict[str, object]:
+    def _state(self):
+        return (self.window_tokens, self.filled, self.prefix_len, self.window_len, self.budget)
+
+    def capture_step(self) -> "torch.cuda.CUDAGraph":
+        """One step of Algorithm 1 (all layers, LM head, confidence / commit / refill) as a CUDA graph.  Every
+        size the step depends on lives in device memory, so one capture serves the whole generation.  One eager
+        step runs first (library and GEMM set-up); the window state is put back afterwards, and what that step
+        staged into the caches lies beyond the committed prefix, where the next step overwrites it."""
+        saved = [t.clone() for t in self._state()]
+        self.step()
+        torch.cuda.synchronize()
+        for t, s0 in zip(self._state(), saved):
+            t.copy_(s0)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.step()
+        for t, s0 in zip(self._state(), saved):
+            t.copy_(s0)
+        self.steps = 0
+        return graph
+
+    def generate(self, max_new_tokens: int, max_steps: int = 1_000_000, use_graph: bool = False) -> Dict[str, object]:
         """Runs until every window is empty.  Returns the committed text per sequence, the number of
-        steps and the prefix cacheability p_cache = N_gen / N_fwd (Eq. 4)."""
+        steps and the prefix cacheability p_cache = N_gen / N_fwd (Eq. 4).  With use_graph the step is
+        captured once and replayed; the host still reads the commits of every step."""
+        if use_graph:
+            return self._generate_graph(max_new_tokens, max_steps)
         self.start(max_new_tokens)
         ys: List[List[int]] = [[] for _ in range(self.B)]
         commits_per_step = []
@@ -186,6 +220,36 @@ class StreamingDecoder:
             cc, ct = self.step()
             cc_h, ct_h = cc.cpu().numpy(), ct.cpu().numpy()
             for b in range(self.B):
+                ys[b].extend(ct_h[b, : cc_h[b]].tolist())
+            commits_per_step.append(int(cc_h.sum()))
+        n_gen = sum(len(y) for y in ys)
+        return dict(y=ys, steps=self.steps, n_fwd=self.n_fwd, p_cache=(n_gen / self.n_fwd if self.n_fwd else 0.0),
+                    commits_per_step=commits_per_step)
+
+    def _generate_graph(self, max_new_tokens: int, max_steps: int) -> Dict[str, object]:
+        self.start(max_new_tokens)
+        graph = self.capture_step()
+        s = self.step_bufs
+        B, W = self.B, self.W
+        # one pinned buffer receives everything the host needs from a step: window_len | count | tokens
+        host = torch.empty(B * (2 + W), dtype=torch.int32).pin_memory()
+        dev = torch.empty(B * (2 + W), dtype=torch.int32, device="cuda")
+        ys: List[List[int]] = [[] for _ in range(B)]
+        commits_per_step = []
+        wl = self.window_len.cpu().numpy()
+        while self.steps < max_steps and int(wl.sum()) > 0:
+            self.n_fwd += int(wl.sum())
+            graph.replay()
+            self.steps += 1
+            dev[:B].copy_(self.window_len)
+            dev[B:2 * B].copy_(s.committed_count)
+            dev[2 * B:].copy_(s.committed_tokens.view(-1))
+            host.copy_(dev, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            h = host.numpy()
+            wl = h[:B].copy()
+            cc_h, ct_h = h[B:2 * B], h[2 * B:].reshape(B, W)
+            for b in range(B):
                 ys[b].extend(ct_h[b, : cc_h[b]].tolist())
             commits_per_step.append(int(cc_h.sum()))
         n_gen = sum(len(y) for y in ys)

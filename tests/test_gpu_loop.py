@@ -71,6 +71,27 @@ def test_tiny_model_sampled_text_is_token_exact(W, tilt, tau, T):
         assert greedy_same < B          # the sampled text is not the greedy text
 
 
+@pytest.mark.parametrize("W,tilt,tau,T", [(8, 8.0, 0.35, 0.0), (4, 6.0, 0.5, 0.7), (1, 0.0, 0.3, 0.0)])
+def test_generation_replayed_from_a_cuda_graph_equals_the_eager_loop(W, tilt, tau, T):
+    """The whole step (layers, LM head, confidence / commit / refill) captured once and replayed: same text,
+    step count and p_cache as the eager loop."""
+    from paper_2512_22737_b200.loop import StreamingDecoder
+    B, P, N = 3, 21, 26
+    wts = make_model(TINY)
+    pt = make_prompts_and_targets(TINY, B, P, N)
+    outs = []
+    for use_graph in (False, True):
+        dec = StreamingDecoder(TINY, wts, batch=B, window=W, max_total_len=P + N, tau=tau, lam=0.1, tilt=tilt,
+                               target=pt["target"], temperature=T, sample_seed=99)
+        dec.prefill(pt["prompt"])
+        outs.append(dec.generate(N, use_graph=use_graph))
+        assert int(dec.step_bufs.status.item()) == 0
+    a, b = outs
+    assert a["y"] == b["y"]
+    assert a["steps"] == b["steps"] and a["n_fwd"] == b["n_fwd"] and a["commits_per_step"] == b["commits_per_step"]
+    assert all(len(y) == N for y in b["y"])
+
+
 @pytest.mark.parametrize("W,tilt,tau", [(4, 8.0, 0.5), (8, 30.0, 0.35)])
 def test_tiny_model_block_wise_baseline_is_token_exact(W, tilt, tau):
     from paper_2512_22737_b200.loop import StreamingDecoder
