@@ -66,3 +66,28 @@ def test_argument_validation_happens_on_the_host():
     # empty batch is a no-op
     cfg0 = w.make_config(batch=0, window=8)
     assert lib.wedlm_reorder(ctypes.byref(cfg0), None, None, None, None, None, None, None, None, None, None, None) == 0
+
+
+def test_newer_entry_points_validate_on_the_host_too():
+    import paper_2512_22737_b200 as w
+    lib = w.load_library()
+    ok = w.make_config(batch=2, window=32, n_q_heads=32, n_kv_heads=8, head_dim=128, page_size=16, max_pages_per_seq=8,
+                       num_pages=32, max_prefix_len=64, vocab=4096, mask_token_id=4095)
+    # whole step from host buffers: sizes, then null pointers
+    assert w.wedlm_step_host_workspace_bytes(ok) > w.wedlm_window_attn_workspace_bytes(ok) + w.wedlm_confidence_workspace_bytes(ok)
+    nulls = [None] * 15
+    assert lib.wedlm_step_host(ctypes.byref(ok), *nulls, None, 0, None, None, None) == -1
+    # Dual-Stream Masking: blocks must own whole pages; n_blocks must match the sequence length
+    assert w.wedlm_dual_stream_workspace_bytes(ok, 4) > 0
+    odd = w.make_config(batch=2, window=24, n_q_heads=32, n_kv_heads=8, head_dim=128, page_size=16, vocab=4096)
+    assert w.wedlm_dual_stream_workspace_bytes(odd, 4) == 0
+    assert lib.wedlm_dual_stream_attn(ctypes.byref(odd), 4, None, None, None, None, None, None, 0, None, None) == -2
+    assert lib.wedlm_dual_stream_construct(ctypes.byref(ok), 4, 200, None, None, None, None, None, None, None) == -1   # 200 > 4 * 32
+    assert lib.wedlm_dual_stream_construct(ctypes.byref(ok), 4, 96, None, None, None, None, None, None, None) == -1    # 96 fits 3 blocks
+    assert lib.wedlm_dual_stream_construct(ctypes.byref(ok), 4, 100, None, None, None, None, None, None, None) == -1   # null pointers
+    # sampling: a negative or non-finite temperature is refused, a positive one enlarges the workspace
+    hot = w.make_config(batch=2, window=32, vocab=4096, sample_temperature=0.5)
+    cold = w.make_config(batch=2, window=32, vocab=4096)
+    assert w.wedlm_confidence_workspace_bytes(hot) > w.wedlm_confidence_workspace_bytes(cold) > 0
+    for bad in (-0.1, float("nan"), float("inf")):
+        assert w.wedlm_confidence_workspace_bytes(w.make_config(batch=2, window=32, vocab=4096, sample_temperature=bad)) == 0
