@@ -19,6 +19,8 @@ Readings of points the paper leaves open:
   * a prediction row of block k sees memory rows at positions < k*B only: not the clean copy of its own
     block, in particular not its own clean token;
   * positions are 0-based.
+Parity unpinned (nothing printed in the paper can confirm them): the first three readings above.  The
+functions themselves are pinned against the rules as stated, by brute force and library special cases.
 """
 from __future__ import annotations
 
