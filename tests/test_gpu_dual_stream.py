@@ -83,7 +83,9 @@ def test_construction_is_bit_exact(name, kw):
 
 
 @pytest.mark.parametrize("impl", ["tensor", "generic"])
-@pytest.mark.parametrize("kw", [{}, dict(seq_len=128, block=16), dict(seq_len=70, block=64, n_q_heads=8, n_kv_heads=8)])
+@pytest.mark.parametrize("kw", [{}, dict(seq_len=128, block=16), dict(seq_len=70, block=64, n_q_heads=8, n_kv_heads=8),
+                                dict(seq_len=100, block=32, n_q_heads=32, n_kv_heads=4, n_seq=1),
+                                dict(seq_len=64, block=16, n_q_heads=16, n_kv_heads=16, n_seq=3)])
 def test_small_sequences_every_row(impl, kw):
     c = DS_CONFIGS["ds_small"].replace(**kw)
     inp = make_dual_stream(c, seed=23)
