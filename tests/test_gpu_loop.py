@@ -45,6 +45,24 @@ def test_tiny_model_text_is_token_exact(W, tilt, tau):
         assert got["steps"] < N
 
 
+def test_tiny_model_step_wise_scheme_w6_is_token_exact():
+    """The evaluation setting of Section 6.1: W = 6, lambda = 0.1, one token per step at the lowest adjusted entropy."""
+    from paper_2512_22737_b200.loop import StreamingDecoder
+    B, P, N, W = 2, 21, 20, 6
+    wts = make_model(TINY)
+    pt = make_prompts_and_targets(TINY, B, P, N)
+    dec = StreamingDecoder(TINY, wts, batch=B, window=W, max_total_len=P + N, tau=float("-inf"), lam=0.1, tilt=5.0,
+                           target=pt["target"])
+    dec.prefill(pt["prompt"])
+    got = dec.generate(N)
+    for b in range(B):
+        ref = mo.decode(wts, TINY, pt["prompt"][b], pt["target"][b], tilt=5.0, window=W, max_new_tokens=N,
+                        conf_mode="entropy", tau=float("-inf"), lam=0.1, maxprob_thr=0.9)
+        assert got["y"][b] == ref["y"]
+        assert all(t["filled"] <= 1 for t in ref["trace"])
+    assert max(got["commits_per_step"]) <= B * W
+
+
 @pytest.mark.parametrize("W,tilt,tau,T", [(4, 6.0, 0.5, 0.7), (8, 4.0, 2.0, 1.0), (8, 8.0, 0.35, 0.1), (1, 2.0, 0.3, 1.5)])
 def test_tiny_model_sampled_text_is_token_exact(W, tilt, tau, T):
     """Sample() at a temperature: the GPU loop and the oracle draw from the same counter-based generator, keyed

@@ -124,6 +124,19 @@ def test_short_windows_and_budget():
     pu.full_parity(cfg, inp, window_len=[8, 5, 3, 3], remaining_budget=[100, 2, 0, 1])
 
 
+def test_step_wise_scheme_fills_exactly_the_lowest_adjusted_entropy():
+    """tau = -inf: no mask ever passes Eq. 11, so every step fills the single mask with the lowest H + lambda d
+    (the unified step-wise scheme of Section 6.1, W = 6, lambda = 0.1)."""
+    import parity_util as pu
+    cfg = _small_qwen(batch=5, window=6, prefix_lo=30, prefix_hi=400, vocab=4096, tau=float("-inf"), lam=0.1, boost=9.0,
+                      boost_prob=0.5, name="stepwise")
+    for seed in (51, 52):
+        r = pu.full_parity(cfg, make_step(cfg, seed=seed))
+        fc = r["step"].filled_count.cpu().numpy()
+        n_mask = cfg.window - r["ref"]["n_filled"]
+        assert ((fc == 1) | (n_mask == 0)).all()
+
+
 def test_maxprob_mode_bf16():
     import parity_util as pu
     cfg = _small_qwen(batch=2, window=16, prefix_lo=40, prefix_hi=80, vocab=4096, conf_mode="maxprob",
