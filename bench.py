@@ -499,6 +499,10 @@ def run_product(args):
                          "traffic_note": "ncu dram bytes of a batch-16 capture scaled by algorithmic bytes",
                          "kernel_ms": attn_ms,
                          "algorithmic_bytes": bts["attn_kernel"]},
+            "step_hbm": {"note": "whole step: K/V and logits streams plus q/out, against the same measured peak",
+                         "algorithmic_bytes": bts["attn_kernel"] + bts["logits_stream"],
+                         "achieved": (bts["attn_kernel"] + bts["logits_stream"]) / (ms * 1e-3) / 1e9, "unit": "GB/s",
+                         "frac": (bts["attn_kernel"] + bts["logits_stream"]) / (ms * 1e-3) / 1e9 / peak},
             "cpu_baseline": cpu,
             "other_workloads": others,
         }
