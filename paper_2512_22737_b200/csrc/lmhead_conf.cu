@@ -176,10 +176,12 @@ lmhead_conf_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
             const int col = ch * 32 + e;
-            float x = __uint_as_float(o[e]);
+            // columns at or beyond n_cols are not part of the row; beyond tile_n they were never written by this
+            // item's MMAs and hold whatever the tensor memory held before (possibly inf): read them as -inf
+            float x = (col < n_cols) ? __uint_as_float(o[e]) : -CUDART_INF_F;
             if (col == tilt_col) x += p.tilt;
-            const float d = fmaxf(fmaf(x, kLog2e, nm), -127.f);
-            const float ex = (col < n_cols) ? ex2_approx(d) : 0.f;
+            const float d = fmaxf(fmaf(x, kLog2e, nm), -127.f);     // -inf and NaN both end at -127, where 2^d flushes to 0
+            const float ex = ex2_approx(d);
             s += ex;
             t = fmaf(d, ex, t);
           }

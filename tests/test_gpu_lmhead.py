@@ -85,3 +85,30 @@ def test_fused_lmhead_rejects_unsupported_shapes():
                                          e, torch.zeros(8, dtype=torch.uint8, device="cuda"), e, None, None, None, None, None,
                                          None, None, None, None, ws)
     assert err.value.code == -2
+
+
+def test_tile_width_that_is_no_multiple_of_32_ignores_stale_tensor_memory():
+    """Regression: with a vocabulary tile of 208 tokens the reduction reads 224 accumulator columns; the last 16 are
+    never written by the tile's MMAs and keep what tensor memory held before.  A first call whose logits overflow
+    to +inf leaves inf in every column of every SM; the second call must still produce finite statistics."""
+    import paper_2512_22737_b200 as w
+    # call 1: 256-wide tiles on all 148 SMs (V = 148 * 256), logits = +inf
+    V1, H, B, W = 148 * 256, 64, 16, 16
+    c1 = w.make_config(batch=B, window=W, vocab=V1, dtype="bf16", mask_token_id=V1 - 1)
+    s1 = w.DecodeStep(c1)
+    i32 = dict(dtype=torch.int32, device="cuda")
+    filled = torch.zeros(B, W, dtype=torch.uint8, device="cuda")
+    tok, pl = torch.zeros(B, W, **i32), torch.zeros(B, **i32)
+    big = torch.full((B, W, H), 1.0e19, dtype=torch.bfloat16, device="cuda")
+    emb1 = torch.full((V1, H), 1.0e19, dtype=torch.bfloat16, device="cuda")
+    s1.reorder(filled, tok, pl)
+    ws1 = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c1), dtype=torch.uint8, device="cuda")
+    w.wedlm_lmhead_confidence_commit(c1, big, emb1, None, 0.0, s1.perm, s1.n_filled, s1.n_commit, tok.clone(), filled.clone(),
+                                     pl.clone(), None, None, s1.argmax, s1.maxprob, s1.entropy, s1.lse, s1.committed_tokens,
+                                     s1.committed_count, s1.filled_count, ws1)
+    torch.cuda.synchronize()
+    # call 2: V = 148 * 208 makes 208 the cheapest tile width; ordinary inputs, compared with the oracle
+    step, ref = _case(16, 16, 148 * 208, 64, seed=77)
+    ent = step.entropy.cpu().numpy()
+    active = ~np.isnan(ref["entropy"])
+    assert np.isfinite(ent[active]).all()
