@@ -206,3 +206,5 @@ def test_fused_lm_head_loop_writes_the_same_text():
         assert outs[1]["y"][b] == pt["target"][b, P:P + N].tolist()
         assert outs[0]["y"][b] == outs[1]["y"][b]
     assert outs[1]["steps"] < N
+    # fp32 logits against bf16-rounded ones can flip a borderline selection, not change the pace of decoding
+    assert abs(outs[0]["steps"] - outs[1]["steps"]) <= 2
