@@ -20,8 +20,14 @@
  *
  * Conventions common to every call
  *   - Every pointer named below is a DEVICE pointer unless it is the config or says "host".
- *     The caller owns all memory; the library allocates and frees nothing and keeps no state
- *     between calls.  Scratch memory is a caller-supplied workspace sized by a query function.
+ *     The caller owns all memory and the library allocates and frees nothing: scratch memory is a
+ *     caller-supplied workspace sized by a query function.  The one exception is
+ *     wedlm_confidence_commit_static, whose scratch is an array inside the library image.
+ *   - No result of one call is remembered for the next.  What the library does keep per process is
+ *     bookkeeping only: a count of the kernels it launched (wedlm_launch_count), the one-shot timing
+ *     hook armed by wedlm_profile_next_attn (per host thread), per-device attributes it asked the
+ *     driver for once (SM count, shared-memory opt-ins) and the device address of the built-in
+ *     scratch array.
  *   - Calls are asynchronous on the CUDA stream passed as `stream` (a cudaStream_t cast to
  *     void*; NULL is the legacy default stream).  No call synchronises with the host.
  *   - All tensors are dense, row-major ("last index fastest") and need 16-byte aligned base
@@ -53,7 +59,7 @@ extern "C" {
 
 /* bits OR-ed into the device status word */
 #define WEDLM_STATUS_BAD_PAGE     1   /* block_table entry outside [0, num_pages)            */
-#define WEDLM_STATUS_BAD_LENGTH   2   /* prefix_len[b] < 0 or prefix_len[b]+W beyond the table */
+#define WEDLM_STATUS_BAD_LENGTH   2   /* prefix_len[b] < 0, > cfg.max_prefix_len, or +W beyond the table */
 #define WEDLM_STATUS_WAIT_EXPIRED 4   /* a bounded on-chip wait gave up (tensor-core path)     */
 
 #define WEDLM_DTYPE_BF16 0
@@ -71,7 +77,7 @@ extern "C" {
 #define WEDLM_ATTN_TENSOR  2   /* tcgen05 + TMA kernel, bf16, head_dim 128, page 16       */
 
 typedef struct wedlm_config {
-  int32_t batch;              /* B  sequences                                              */
+  int32_t batch;              /* B  sequences (any count a 1-D grid can index)             */
   int32_t window;             /* W  slots per sequence (1..1024)                           */
   int32_t n_q_heads;          /* Hq                                                        */
   int32_t n_kv_heads;         /* Hkv, divides Hq; query head h reads KV head h / (Hq/Hkv)  */
@@ -89,7 +95,11 @@ typedef struct wedlm_config {
   float   lambda;             /* distance penalty of Eq. 11                                */
   float   maxprob_thr;
   int32_t mask_token_id;      /* token id written into fresh mask slots                    */
-  int32_t max_prefix_len;     /* host-known upper bound of prefix_len[b]; sizes the grid   */
+  int32_t max_prefix_len;     /* host-known upper bound of prefix_len[b]: sizes the key split and the  */
+                              /* workspace.  A prefix_len[b] above it (the device value moved on while */
+                              /* the host bound did not) is treated as max_prefix_len by the attention */
+                              /* kernels and flagged WEDLM_STATUS_BAD_LENGTH; nothing is written out   */
+                              /* of bounds, the rows of that sequence are then wrong.                  */
   int32_t attn_impl;          /* WEDLM_ATTN_*                                              */
   int32_t commit_mode;        /* WEDLM_COMMIT_*                                            */
   float   sample_temperature; /* 0: Sample() is the arg-max; > 0: one draw from softmax(l/T) */
@@ -103,7 +113,8 @@ const char* wedlm_strerror(int code);
 /* Library version, major*10000 + minor*100 + patch. */
 int wedlm_version(void);
 
-/* Measurement aids (no counterpart in the paper).
+/* Measurement aids and self-test: not part of the decoding path, no counterpart in the paper, and no
+ * stability promise (they may change between versions without the call signatures above them changing).
  * wedlm_launch_count: kernels launched through this library by the calling process so far.
  * wedlm_profile_next_attn: the next wedlm_window_attn call made by the calling host thread records
  *   the two CUDA events (cudaEvent_t cast to void*, host handles, either may be NULL) on its stream
@@ -269,8 +280,11 @@ int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, co
  *   - Limit: wedlm_confidence_workspace_bytes(cfg) must not exceed WEDLM_STATIC_SCRATCH_BYTES
  *     (4 MiB = 262144 chunk partials; batch*window*ceil(vocab/8192) for bf16, /4096 for fp32).
  *     Larger problems return WEDLM_ERR_STATIC_SCRATCH and launch nothing.
- *   - The first call on each device looks up the array's device address (one runtime query, no
- *     allocation) with that device current; make that first call before starting any stream capture.
+ *   - The first call on each device looks up the array's device address with that device current.
+ *     The array is part of the library's device image, which the CUDA runtime places in device memory
+ *     when it loads the module on that device; with lazy module loading that can be this first call.
+ *     Make the first call early (at start-up, before memory becomes scarce) and before starting any
+ *     stream capture.  Later calls query nothing and allocate nothing.
  *   - All calls on a device share the one array.  It keeps whatever the previous call left there;
  *     this routine needs none of it zeroed.  Two calls whose kernels can overlap on the GPU (different
  *     streams, no ordering between them) race on the array: serialise them.

@@ -1,6 +1,5 @@
 // C ABI of the WeDLM step library: argument validation, workspace planning, kernel dispatch.
 #include <atomic>
-#include <cstdlib>
 
 #include "common.cuh"
 
@@ -16,6 +15,24 @@ thread_local cudaEvent_t t_ev_after = nullptr;
 
 namespace wedlm {
 void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+int device_sm_count() {
+  constexpr int kFallbackSms = 148;
+  static std::atomic<int> cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return kFallbackSms; }
+  if (dev >= 0 && dev < 64) {
+    const int have = cached[dev].load(std::memory_order_relaxed);
+    if (have > 0) return have;
+  }
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+    cudaGetLastError();
+    return kFallbackSms;
+  }
+  if (dev >= 0 && dev < 64) cached[dev].store(sms, std::memory_order_relaxed);
+  return sms;
+}
 }  // namespace wedlm
 
 namespace {
@@ -54,6 +71,7 @@ Shape make_shape(const wedlm_config_t* c) {
   s.G = c->n_kv_heads > 0 ? c->n_q_heads / c->n_kv_heads : 1;
   s.page = c->page_size; s.max_pages = c->max_pages_per_seq; s.num_pages = c->num_pages; s.V = c->vocab;
   s.dtype = c->dtype; s.rope_style = c->rope_style; s.theta = c->rope_theta; s.commit_mode = c->commit_mode;
+  s.max_prefix = c->max_prefix_len;
   s.scale = c->softmax_scale > 0.f ? c->softmax_scale : 1.0f / sqrtf((float)c->head_dim);
   return s;
 }
@@ -81,7 +99,7 @@ AttnPlan plan_attention(const wedlm_config_t* c) {
     // (2 per SM) balances well without splitting the keys, and then no partials exist at all.  With
     // fewer units the keys are split just far enough to fill the slots: the smallest split count
     // whose last wave is at least 85 % full, chunks no shorter than 256 keys.
-    const long long slots = 2LL * 148;
+    const long long slots = 2LL * device_sm_count();
     long long cap = total / 256 > 1 ? total / 256 : 1;
     if (cap > 64) cap = 64;
     S = 1;
@@ -95,13 +113,12 @@ AttnPlan plan_attention(const wedlm_config_t* c) {
         if (eff >= 0.85) { S = cand; break; }
       }
     }
-    if (const char* e = getenv("WEDLM_ATTN_SPLITS")) { long long v = atoll(e); if (v > 0) S = v > cap ? cap : v; }
     chunk = (total + S - 1) / S;
     chunk = (chunk + 63) / 64 * 64;
   } else {
     const long long n_rb = (c->window + 15) / 16;
     const long long units = (long long)c->batch * c->n_q_heads * n_rb;
-    long long want = units > 0 ? (148LL * 4 + units - 1) / units : 1;      // a few blocks per SM
+    long long want = units > 0 ? (4LL * device_sm_count() + units - 1) / units : 1;      // a few blocks per SM
     long long cap = total / 256 > 1 ? total / 256 : 1;                      // keep chunks >= 256 keys
     S = want < 1 ? 1 : (want > cap ? cap : want);
     chunk = (total + S - 1) / S;

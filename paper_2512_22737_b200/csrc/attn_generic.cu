@@ -12,7 +12,7 @@ namespace wedlm {
 constexpr int kRB = 16;         // query rows per block
 constexpr int kThreads = 128;
 
-// grid: x = key split, y = h * n_rowblocks + rb, z = b
+// 1-D grid, block index = (b * Hq * n_rowblocks + h * n_rowblocks + rb) * n_splits + split
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 attn_generic_kernel(Shape s, int n_splits, int chunk, const T* __restrict__ q_rot, const T* __restrict__ k_cache,
@@ -33,12 +33,14 @@ attn_generic_kernel(Shape s, int n_splits, int chunk, const T* __restrict__ q_ro
   float* ls = ms + kRB;                   // [kRB] running sum
 
   const int tid = threadIdx.x;
-  const int split = blockIdx.x, b = blockIdx.z;
   const int n_rb = (s.W + kRB - 1) / kRB;
-  const int h = blockIdx.y / n_rb, rb = blockIdx.y - h * n_rb;
+  const unsigned per_seq = (unsigned)(s.Hq * n_rb * n_splits);
+  const int b = (int)(blockIdx.x / per_seq);
+  const int in_seq = (int)(blockIdx.x - (unsigned)b * per_seq);
+  const int split = in_seq % n_splits, hrb = in_seq / n_splits;
+  const int h = hrb / n_rb, rb = hrb - h * n_rb;
   const int g = h / s.G;
-  int P = prefix_len[b];
-  if (P < 0) { if (status && tid == 0) atomicOr(status, WEDLM_STATUS_BAD_LENGTH); P = 0; }
+  const int P = checked_prefix(prefix_len, b, s.max_prefix, status, tid == 0);
   const int total = P + s.W;
   const int n_valid = (total + chunk - 1) / chunk;
   if (split >= n_valid) return;
@@ -157,7 +159,7 @@ attn_merge_kernel(Shape s, int n_splits, int chunk, const int32_t* __restrict__ 
   if (warp >= s.B * rows_per_seq) return;
   const int b = warp / rows_per_seq, rem = warp - b * rows_per_seq;
   const int h = rem / s.W, i = rem - h * s.W;                       // partial rows are ordered (b, h, i)
-  const int P = max(prefix_len[b], 0);
+  const int P = checked_prefix(prefix_len, b, s.max_prefix, nullptr, false);      // same clamp as the attention kernels
   const int n_valid = min(n_splits, (P + s.W + chunk - 1) / chunk);
   if (n_valid <= 1) return;
   const size_t prow = (size_t)warp * n_splits;
@@ -191,7 +193,8 @@ static int launch_generic_t(const Shape& s, const AttnPlan& plan, const void* q_
                             const void* v_cache, const int32_t* block_table, const int32_t* prefix_len, void* out,
                             float* part_o, float* part_ml, int32_t* status, cudaStream_t st) {
   const int n_rb = (s.W + kRB - 1) / kRB;
-  dim3 grid(plan.n_splits, s.Hq * n_rb, s.B);
+  const long long blocks = (long long)plan.n_splits * s.Hq * n_rb * s.B;
+  if (blocks > 0x7fffffffLL) return WEDLM_ERR_UNSUPPORTED;
   size_t smem = sizeof(float) * ((size_t)kRB * D + (size_t)s.page * (D + 1) + (size_t)s.page * D +
                                  (size_t)kRB * s.page + 3 * kRB);
   auto kern = attn_generic_kernel<T, D>;
@@ -199,7 +202,7 @@ static int launch_generic_t(const Shape& s, const AttnPlan& plan, const void* q_
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return WEDLM_ERR_CUDA;
   }
-  kern<<<grid, kThreads, smem, st>>>(s, plan.n_splits, plan.chunk, (const T*)q_rot, (const T*)k_cache,
+  kern<<<(unsigned)blocks, kThreads, smem, st>>>(s, plan.n_splits, plan.chunk, (const T*)q_rot, (const T*)k_cache,
                                      (const T*)v_cache, block_table, prefix_len, (T*)out, part_o, part_ml, status);
   count_launch();
   return cuda_ok(cudaGetLastError());

@@ -44,12 +44,11 @@ constexpr uint32_t kStageBytes = 16384;
 constexpr uint32_t kHalfKV = 8192;
 constexpr uint32_t kHalfQ = 16384;
 
-// (the TRACE macro below is empty in normal builds)
 enum Bar { Q_FULL = 0, K_FULL0, K_FULL1, V_FULL0, V_FULL1, S_FULL0, S_FULL1, O_DONE, P_READY, K_FREE0, K_FREE1,
            V_FREE0, V_FREE1, N_BARS };
 
 struct TensorAttnParams {
-  int B, W, Hq, Hkv, G, W_t, n_mtiles, n_splits, chunk, max_pages, num_pages;
+  int B, W, Hq, Hkv, G, W_t, n_mtiles, n_splits, chunk, max_pages, num_pages, max_prefix;
   float scale_log2;          // softmax scale * log2(e)
   const int32_t* block_table;
   const int32_t* prefix_len;
@@ -60,30 +59,21 @@ struct TensorAttnParams {
   int32_t* status;
 };
 
-#ifdef WEDLM_ATTN_TRACE
-}  // namespace
-// Debug builds only: per-tile timestamps of one CTA, [role][tile][event].
-__device__ long long g_attn_trace[4 * 256 * 8];
-namespace {
-#define TRACE(role, t, ev) do { if (trace_on && (unsigned)(t) < 256u) g_attn_trace[((role) * 256 + (t)) * 8 + (ev)] = clock64(); } while (0)
-#else
-#define TRACE(role, t, ev) do { } while (0)
-#endif
-
 using namespace ptx;
 
-// grid: x = split * n_mtiles + mtile, y = kv head, z = sequence
+// 1-D grid, block index = (sequence rank * Hkv + kv head) * (n_splits * n_mtiles) + split * n_mtiles + mtile
 __global__ void __launch_bounds__(kThreadsT, 2)
 attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const TensorAttnParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int split = blockIdx.x / p.n_mtiles, mtile = blockIdx.x - split * p.n_mtiles;
-  const int g = blockIdx.y;
-  const int b = p.order ? p.order[blockIdx.z] : (int)blockIdx.z;     // longest sequences are dispatched first
+  const int per_head = p.n_splits * p.n_mtiles;
+  const int unit = (int)(blockIdx.x / (unsigned)per_head), in_head = (int)(blockIdx.x - (unsigned)unit * per_head);
+  const int split = in_head / p.n_mtiles, mtile = in_head - split * p.n_mtiles;
+  const int rank = unit / p.Hkv, g = unit - rank * p.Hkv;
+  const int b = p.order ? p.order[rank] : rank;                      // longest sequences are dispatched first
 
-  int P = p.prefix_len[b];
-  if (P < 0) { if (p.status && tid == 0) atomicOr(p.status, WEDLM_STATUS_BAD_LENGTH); P = 0; }
+  const int P = checked_prefix(p.prefix_len, b, p.max_prefix, p.status, tid == 0);
   const int total = P + p.W;
   const int n_valid = (total + p.chunk - 1) / p.chunk;
   if (split >= n_valid) return;
@@ -99,9 +89,6 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const int h = g * p.G + r % p.G;                           // query head
   const bool row_valid = (tid < 128) && (i_row < p.W);
   const float c = p.scale_log2;
-#ifdef WEDLM_ATTN_TRACE
-  const bool trace_on = (blockIdx.x == 0 && blockIdx.y == 3 && blockIdx.z == 0) && (lane == 0);
-#endif
 
   if (T == 0) {
     // nothing visible in this chunk for these rows: an empty partial (only possible when n_splits > 1)
@@ -160,7 +147,6 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           const uint64_t bd = make_desc(sbase + kOffK + st * kStageBytes + (kk >> 2) * kHalfKV + (kk & 3) * 32u, 16u, 1024u);
           umma(tmem_S + st * 64u, ad, bd, idesc_qk, kk > 0);
         }
-        TRACE(0, t - 1, 6);
         umma_commit(bar(S_FULL0 + st));
         umma_commit(bar(K_FREE0 + st));
       };
@@ -171,19 +157,14 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t st = (uint32_t)t & 1u, ph = ((uint32_t)t >> 1) & 1u;
         if (t + 1 < T) {
           // S[(t+1)&1] was last read by the softmax of tile t-1, whose P_READY we saw one iteration ago
-          TRACE(0, t, 0);
           ok = mbar_wait(bar(K_FULL0 + (st ^ 1u)), ((uint32_t)(t + 1) >> 1) & 1u);
           if (!ok) break;
-          TRACE(0, t, 1);
           issue_qk(t + 1);
-          TRACE(0, t, 2);
         }
         ok = mbar_wait(bar(P_READY), (uint32_t)t & 1u);
         if (!ok) break;
-        TRACE(0, t, 3);
         ok = mbar_wait(bar(V_FULL0 + st), ph);
         if (!ok) break;
-        TRACE(0, t, 4);
         tc_fence_after();
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -193,7 +174,6 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         umma_commit(bar(O_DONE));
         umma_commit(bar(V_FREE0 + st));
-        TRACE(0, t, 5);
       }
       if (!ok) {
         *abort_flag = 1;
@@ -242,14 +222,11 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       const uint32_t st = (uint32_t)t & 1u;
       const int y = y_next;
       if (t + 1 < T) y_next = page_row(t + 1);              // table entry of the next tile, used one iteration later
-      TRACE(is_k ? 1 : 3, t, 0);
       if (t >= 2) ok = wait_all(bar(free0 + st), ((uint32_t)(t - 2) >> 1) & 1u);
       if (!ok) break;
-      TRACE(is_k ? 1 : 3, t, 1);
       if (lane == 0) mbar_expect_tx(bar(full0 + st), kStageBytes);
       __syncwarp();
       if (lane < 8) tma_load_2d(stage0 + st * kStageBytes + lane_dst, map, half * 64, y, bar(full0 + st));
-      TRACE(is_k ? 1 : 3, t, 2);
     }
     if (!ok && lane == 0) {
       *abort_flag = 1;
@@ -264,10 +241,8 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     bool ok = true;
     for (int t = 0; t < T; ++t) {
       const uint32_t st = (uint32_t)t & 1u, ph = ((uint32_t)t >> 1) & 1u;
-      TRACE(2, t, 0);
       ok = mbar_wait(bar(S_FULL0 + st), ph);
       if (!ok) break;
-      TRACE(2, t, 1);
       tc_fence_after();
       uint32_t raw[64];
       {
@@ -277,7 +252,6 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tmem_ld32(tmem_S + lane_sel + st * 64u + 32u, hi);
         tmem_wait_ld();
       }
-      TRACE(2, t, 2);
       const int tile0 = kv_begin + t * kTileN;
       const bool need_mask = tile0 + kTileN > min(P + slot0 + 1, kv_end);   // block-uniform
       float m_tile;
@@ -302,7 +276,6 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         m_tile = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
       }
-      TRACE(2, t, 7);
       // lazy reference: only move it when the maximum grew by more than 2^kLazyRescaleLog2
       float alpha = 1.f;
       bool moved = false;
@@ -336,11 +309,9 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
       l = l * alpha + (sum + sum2);
       // P buffer and O are free / stable once P V_{t-1} has completed
-      TRACE(2, t, 3);
       if (t > 0) {
         ok = mbar_wait(bar(O_DONE), (uint32_t)(t - 1) & 1u);
         if (!ok) break;
-        TRACE(2, t, 4);
         tc_fence_after();
         if (__any_sync(0xffffffffu, moved)) {
 #pragma unroll 1
@@ -375,11 +346,9 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           *reinterpret_cast<uint4*>(vst + (ch >> 3) * kHalfKV + row * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
         }
       }
-      TRACE(2, t, 5);
       fence_async_smem();
       tc_fence_before();
       mbar_arrive(bar(P_READY));
-      TRACE(2, t, 6);
     }
     if (ok) ok = mbar_wait(bar(O_DONE), (uint32_t)(T - 1) & 1u);
     if (!ok) {
@@ -388,6 +357,7 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     } else {
       tc_fence_after();
       const bool final_out = n_valid == 1;        // the only chunk of this sequence: write the result itself
+                                                  // (n_valid <= n_splits because P is clamped to the planned bound)
       const float inv = l > 0.f ? 1.f / l : 0.f;
       const size_t orow = (((size_t)b * p.W + i_row) * p.Hq + h) * kD;
       const size_t prow = (((size_t)b * p.Hq + h) * p.W + i_row) * p.n_splits + split;
@@ -475,14 +445,6 @@ int launch_wait_expiry_selftest(uint32_t max_polls, int32_t* status, cudaStream_
   return cuda_ok(cudaGetLastError());
 }
 
-#ifdef WEDLM_ATTN_TRACE
-}  // namespace wedlm
-extern "C" int wedlm_debug_read_attn_trace(long long* host_dst) {
-  return cudaMemcpyFromSymbol(host_dst, wedlm::g_attn_trace, sizeof(long long) * 4 * 256 * 8) == cudaSuccess ? 0 : -4;
-}
-namespace wedlm {
-#endif
-
 bool attn_tensor_supported(const wedlm_config_t* c) {
   if (c->dtype != WEDLM_DTYPE_BF16 || c->head_dim != kD || c->page_size != kPage) return false;
   const int G = c->n_q_heads / c->n_kv_heads;
@@ -526,6 +488,7 @@ int launch_attn_tensor(const Shape& s, const AttnPlan& plan, const void* q_rot, 
   TensorAttnParams p;
   p.B = s.B; p.W = s.W; p.Hq = s.Hq; p.Hkv = s.Hkv; p.G = s.G; p.W_t = W_t; p.n_mtiles = n_mtiles;
   p.n_splits = plan.n_splits; p.chunk = plan.chunk; p.max_pages = s.max_pages; p.num_pages = s.num_pages;
+  p.max_prefix = s.max_prefix;
   p.scale_log2 = s.scale * 1.4426950408889634f;
   p.block_table = block_table; p.prefix_len = prefix_len; p.order = order;
   p.out = (__nv_bfloat16*)out; p.part_o = part_o; p.part_ml = part_ml; p.status = status;
@@ -541,8 +504,9 @@ int launch_attn_tensor(const Shape& s, const AttnPlan& plan, const void* q_rot, 
       if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
   }
-  dim3 grid(plan.n_splits * n_mtiles, s.Hkv, s.B);
-  attn_tensor_kernel<<<grid, kThreadsT, kSmemBytes, st>>>(tm_q, tm_k, tm_v, p);
+  const long long blocks = (long long)plan.n_splits * n_mtiles * s.Hkv * s.B;
+  if (blocks > 0x7fffffffLL) return WEDLM_ERR_UNSUPPORTED;
+  attn_tensor_kernel<<<(unsigned)blocks, kThreadsT, kSmemBytes, st>>>(tm_q, tm_k, tm_v, p);
   count_launch();
   return cuda_ok(cudaGetLastError());
 }

@@ -13,8 +13,24 @@ struct Shape {
   int B, W, Hq, Hkv, D, G;
   int page, max_pages, num_pages, V;
   int dtype, rope_style, commit_mode;
+  int max_prefix;      // host-known bound of prefix_len[b]: the key split and the workspace are sized for it
   float theta, scale;
 };
+
+// prefix_len[b] as the attention kernels use it.  The value is device data and may have moved past the bound
+// the launch was planned for (or be negative): such a value is flagged in *status by the `report` thread and
+// clamped into [0, max_prefix], so that every index derived from it stays inside the planned key chunks and
+// the partial buffers.  The merge kernel applies the same clamp (without reporting) and so agrees on the
+// number of chunks.
+__device__ __forceinline__ int checked_prefix(const int32_t* __restrict__ prefix_len, int b, int max_prefix,
+                                              int32_t* status, bool report) {
+  int P = prefix_len[b];
+  if (P < 0 || P > max_prefix) {
+    if (report && status) atomicOr(status, WEDLM_STATUS_BAD_LENGTH);
+    P = P < 0 ? 0 : max_prefix;
+  }
+  return P;
+}
 
 __device__ __forceinline__ float ld_as_float(const float* p, size_t i) { return p[i]; }
 __device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p, size_t i) { return __bfloat162float(p[i]); }
@@ -108,6 +124,10 @@ int launch_window_refill(const Shape& s, const wedlm_config_t* cfg, const int32_
                          int32_t* committed_tokens, int32_t* committed_count, cudaStream_t st);
 
 inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? WEDLM_OK : WEDLM_ERR_CUDA; }
+
+// Multiprocessor count of the current device, asked once per device ordinal; 148 (B200) when no device
+// can be asked, which only happens in size queries made on a host without a GPU.
+int device_sm_count();
 
 // Number of kernels this process has launched through the library (reported by wedlm_launch_count).
 void count_launch(int n = 1);

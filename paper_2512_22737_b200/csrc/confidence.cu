@@ -722,18 +722,14 @@ int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* log
     if (vec) {
       const size_t smem = (size_t)kStreamStages * kStreamChunk * 2 + kStreamStages * 24;
       static bool attr_done[64] = {};
-      static int sm_count[64] = {};
-      int dev = 0, sms = 148;
+      int dev = 0;
       if (cudaGetDevice(&dev) != cudaSuccess) return WEDLM_ERR_CUDA;
       if (dev < 0 || dev >= 64 || !attr_done[dev]) {
         if (cudaFuncSetAttribute(conf_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
           return WEDLM_ERR_CUDA;
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (dev >= 0 && dev < 64) { attr_done[dev] = true; sm_count[dev] = sms; }
-      } else {
-        sms = sm_count[dev];
+        if (dev >= 0 && dev < 64) attr_done[dev] = true;
       }
-      long long grid = (long long)sms * kStreamBlocksPerSM;
+      long long grid = (long long)device_sm_count() * kStreamBlocksPerSM;
       if (grid > blocks) grid = blocks;
       conf_stream_kernel<<<(unsigned)grid, kStreamThreads + 32, smem, st>>>(s.W, s.V, n_chunks, blocks, (const T*)logits, n_filled,
                                                                       window_len, part);
@@ -757,9 +753,7 @@ int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* log
   if (rc != WEDLM_OK || !sampling) return rc;
   // third pass: draw the tokens of the rows selected above
   const SampleWs sw = carve_sample_ws(sample_ws, rows);
-  int dev = 0, sms = 148;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  long long grid = (long long)sms * 8;
+  long long grid = (long long)device_sm_count() * 8;
   if (grid > blocks) grid = blocks;
   const float inv_t = (float)(1.0 / (double)cfg->sample_temperature);
   if (s.dtype == WEDLM_DTYPE_BF16) {

@@ -239,19 +239,15 @@ int launch_lmhead_conf(const Shape& s, int hidden, const void* hidden_states, co
   auto encode = lm_get_encode();
   if (!encode) return WEDLM_ERR_CUDA;
   const int R = s.B * s.W;
-  int sms = 148;
+  const int sms = device_sm_count();
   {
     static bool attr_done[64] = {};
-    static int sm_count[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return WEDLM_ERR_CUDA;
     if (dev < 0 || dev >= 64 || !attr_done[dev]) {
       if (cudaFuncSetAttribute(lmhead_conf_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmSmem) != cudaSuccess)
         return WEDLM_ERR_CUDA;
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-      if (dev >= 0 && dev < 64) { attr_done[dev] = true; sm_count[dev] = sms; }
-    } else {
-      sms = sm_count[dev];
+      if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
   }
   const int row_chunks = (R + kLmRows - 1) / kLmRows;

@@ -29,7 +29,7 @@ __device__ __forceinline__ void rotate8(const uint4& a, const uint4& c, const fl
   oc = make_uint4(rc[0], rc[1], rc[2], rc[3]);
 }
 
-// grid (W, B); one block per (physical row i, sequence b).  Angles are formed in double so that
+// grid (B, W); one block per (sequence b, physical row i).  Angles are formed in double so that
 // positions of tens of thousands keep full fp32 accuracy after the range reduction.
 template <typename T>
 __global__ void __launch_bounds__(128)
@@ -39,7 +39,7 @@ rope_stage_kernel(Shape s, const InvFreq inv_freq, const T* __restrict__ q, cons
                   const int32_t* __restrict__ pos_ids, const int32_t* __restrict__ count,
                   int32_t* __restrict__ kv_slot_idx, int32_t* __restrict__ order, int32_t* status) {
   extern __shared__ float cs_sn[];  // [D/2] cos, [D/2] sin
-  const int i = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int b = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
   const int D = s.D, half = D / 2;
   float* cs = cs_sn;
   float* sn = cs_sn + half;
@@ -152,7 +152,7 @@ rope_stage_kernel(Shape s, const InvFreq inv_freq, const T* __restrict__ q, cons
 int launch_rope_stage(const Shape& s, const void* q, const void* k, const void* v, void* q_rot, void* k_cache,
                       void* v_cache, const int32_t* block_table, const int32_t* prefix_len, const int32_t* pos_ids,
                       const int32_t* count, int32_t* kv_slot_idx, int32_t* order, int32_t* status, cudaStream_t st) {
-  dim3 grid(s.W, s.B);
+  dim3 grid(s.B, s.W);      // W <= 1024 fits gridDim.y; the batch may be large (dual-stream units)
   size_t smem = (size_t)s.D * sizeof(float);
   InvFreq inv_freq;
   for (int d = 0; d < s.D / 2; ++d) inv_freq.v[d] = pow((double)s.theta, -2.0 * (double)d / (double)s.D);

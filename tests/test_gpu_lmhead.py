@@ -45,17 +45,18 @@ def _case(B, W, V, H, seed, boost=6.0, window_len=None, budget=None, commit_mode
     d["window_len"], d["remaining_budget"] = wl, bud
     # arg-max: exact unless the two best logits of the row are within the 1e-3 band
     am = step.argmax.cpu().numpy()
-    near_tie = 0
+    near_tie = set()
     for b in range(B):
         for i in range(W):
             if ref["argmax"][b, i] >= 0 and am[b, i] != ref["argmax"][b, i]:
                 top2 = np.sort(logits[b, i])[-2:]
                 assert top2[1] - top2[0] <= 1e-3, (b, i, am[b, i], ref["argmax"][b, i], top2)
-                near_tie += 1
+                near_tie.add(b)
                 ref["argmax"][b, i] = am[b, i]
-    assert near_tie == 0 or near_tie <= 2
-    if near_tie == 0:
-        pu.check_confidence_and_commit(cfg, step, d, inp, ref, window_len)
+    assert len(near_tie) <= 2
+    # a sequence with a near-tie may have filled a different (equally good) token: only its fills are skipped,
+    # every statistic of every row and everything else about its window are still compared
+    pu.check_confidence_and_commit(cfg, step, d, inp, ref, window_len, tie_seqs=near_tie)
     return step, ref
 
 

@@ -1,8 +1,7 @@
 """GPU-vs-oracle parity of the whole step, through the C-ABI binding.
 
-Small cases are compared element by element; the full-size serving and long-context workloads
-are compared on every integer output and on sampled attention vectors / confidence rows the
-oracle can compute one at a time."""
+Small cases and the full-size serving and long-context workloads alike are compared element by
+element: every integer output, every confidence row, every attention output vector."""
 import numpy as np
 import pytest
 import torch
@@ -271,42 +270,106 @@ def test_kv_append_alone_and_window_refill_alone():
         assert d["prefix_len"][b].item() == inp["prefix_len"][b] + n
 
 
-def _sampled_full_size(cfg_name, impl, n_attn=24, n_rows=24):
+_FULL_SIZE_REF = {}
+
+
+def _full_size_reference(cfg_name):
+    """Inputs and the oracle's whole step (attention of every row included) of a full-size workload,
+    computed once per test session and shared by the two attention implementations."""
     import parity_util as pu
-    cfg = get_config(cfg_name)
-    inp = make_step(cfg)
+    if cfg_name not in _FULL_SIZE_REF:
+        cfg = get_config(cfg_name)
+        inp = make_step(cfg)
+        _FULL_SIZE_REF[cfg_name] = (cfg, inp, pu.oracle_step(cfg, inp, with_attention=True))
+    return _FULL_SIZE_REF[cfg_name]
+
+
+def _full_size(cfg_name, impl):
+    """The benchmark's own workload at its full size, in the launch configuration the benchmark times:
+    every integer output, every confidence row, every attention output vector (all B*W*Hq of them) and
+    every staged cache row are compared with the oracle."""
+    import parity_util as pu
+    cfg, inp, ref = _full_size_reference(cfg_name)
     step, d = pu.run_gpu_step(cfg, inp, attn_impl=impl)
-    ref = pu.oracle_step(cfg, inp, with_attention=False)        # integers + confidence on every mask row
     pu.check_reorder(step, ref)
-    np.testing.assert_array_equal(step.kv_slot_idx.cpu().numpy(), ref["kv_slot_idx"])
-    assert int(step.status.item()) == 0
+    worst = pu.check_attention(cfg, step, d, inp, ref)
     excluded = pu.check_confidence_and_commit(cfg, step, d, inp, ref)
+    print(cfg_name, impl, "worst attention error over all vectors", worst, "excluded sequences", excluded)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_cfg3_batched_serving_full_size_every_vector(impl):
+    _full_size("cfg3_batched", impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_cfg4_long_context_full_size_every_vector(impl):
+    _full_size("cfg4_long", impl)
+
+
+def test_reorder_all_1024_patterns_of_a_10_slot_window_in_one_launch():
+    """Every fill pattern of W = 10 as one batch of 1024 sequences: permutation, inverse, position ids,
+    scattered tokens, filled count and commit length bit-exact against the oracle (Eq. 5-6, Algorithm 1)."""
+    import itertools
+    import paper_2512_22737_b200 as w
+    W = 10
+    pats = np.array(list(itertools.product([0, 1], repeat=W)), dtype=np.uint8)
+    B = len(pats)
+    rng = np.random.default_rng(10)
+    P = rng.integers(0, 5000, size=B).astype(np.int32)
+    toks = rng.integers(0, 150000, size=(B, W)).astype(np.int32)
+    for window_len in (None, rng.integers(0, W + 1, size=B).astype(np.int32)):
+        ref = orc.reorder(pats, P, window_len=window_len)
+        c = w.make_config(batch=B, window=W)
+        step = w.DecodeStep(c)
+        wl = None if window_len is None else torch.tensor(window_len, device="cuda")
+        step.reorder(torch.tensor(pats, device="cuda"), torch.tensor(toks, device="cuda"), torch.tensor(P, device="cuda"), wl)
+        torch.cuda.synchronize()
+        for name in ("perm", "inv_perm", "pos_ids", "n_filled", "n_commit"):
+            np.testing.assert_array_equal(getattr(step, name).cpu().numpy(), ref[name], err_msg=name)
+        np.testing.assert_array_equal(step.tokens_phys.cpu().numpy(), np.take_along_axis(toks, ref["perm"], axis=1))
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("planned,actual", [(100, 600), (2000, 5000), (2000, 2001)])
+def test_prefix_beyond_the_planned_bound_is_flagged_and_writes_nothing_out_of_bounds(impl, planned, actual):
+    """prefix_len lives on the device and may run ahead of the host's max_prefix_len.  The key split and the
+    workspace were sized from the host bound, so the kernels clamp the device value to it, set
+    WEDLM_STATUS_BAD_LENGTH and stay inside the workspace: guard bytes behind it keep their pattern, the
+    output stays finite, and a second sequence that respects the bound is still computed correctly."""
+    import paper_2512_22737_b200 as w
+    import parity_util as pu
+    cfg = _small_qwen(batch=2, window=8, prefix_lo=planned, prefix_hi=planned, vocab=1000, name="overrun")
+    inp = make_step(cfg, seed=planned + actual)
+    ref = pu.oracle_step(cfg, inp)
+    d = pu.device_inputs(inp)
+    # the table of sequence 0 also covers the larger prefix: the extra entries all name a spare page that no
+    # sequence owns, so the rows staged at the overrun position land there and disturb nothing
+    n_pages_needed = (actual + cfg.window + 15) // 16
+    pool = inp["k_cache"].shape[0]
+    owned = set(inp["block_table"][inp["block_table"] >= 0].tolist())
+    spare = next(pg for pg in range(pool) if pg not in owned)
+    n_have = inp["block_table"].shape[1]
+    table = torch.zeros(2, max(n_pages_needed, n_have), dtype=torch.int32, device="cuda")
+    table[:, :n_have] = d["block_table"].clamp(min=0)
+    table[0, n_have:] = spare
+    c = w.config_for(cfg, max_pages_per_seq=table.shape[1], num_pages=pool, max_prefix_len=planned, attn_impl=impl)
+    step = w.DecodeStep(c)
+    need = w.wedlm_window_attn_workspace_bytes(c)
+    guard = 1 << 16
+    ws_full = torch.full((need + guard,), 0xAB, dtype=torch.uint8, device="cuda")
+    prefix = d["prefix_len"].clone()
+    prefix[0] = actual
+    step.reorder(d["filled"], d["window_tokens"], d["prefix_len"])          # position ids of the planned prefix
+    w.wedlm_window_attn(c, d["q"], d["k"], d["v"], d["k_cache"], d["v_cache"], table, prefix, step.pos_ids, step.out,
+                        step.kv_slot_idx, ws_full[:need], step.status)
+    torch.cuda.synchronize()
+    assert int(step.status.item()) & w.binding.WEDLM_STATUS_BAD_LENGTH
+    assert not int(step.status.item()) & w.binding.WEDLM_STATUS_WAIT_EXPIRED
+    assert bool((ws_full[need:] == 0xAB).all()), "bytes behind the workspace were overwritten"
     got = pu.bf16_from_device(step.out)
     assert np.isfinite(got).all()
-    rng = np.random.default_rng(0)
-    B, W, Hq = cfg.batch, cfg.window, cfg.n_q_heads
-    worst = 0.0
-    samples = [(int(rng.integers(B)), int(rng.integers(W)), int(rng.integers(Hq))) for _ in range(n_attn)]
-    samples += [(0, 0, 0), (B - 1, W - 1, Hq - 1), (int(np.argmax(inp["prefix_len"])), W - 1, 0),
-                (int(np.argmin(inp["prefix_len"])), 0, Hq - 1)]
-    for (b, i, h) in samples:
-        want = orc.window_attention_row(inp["q"], inp["k"], inp["v"], inp["k_cache"], inp["v_cache"],
-                                        inp["block_table"], inp["prefix_len"], ref["pos_ids"], b, i, h,
-                                        theta=cfg.rope_theta)
-        err = float(np.abs(got[b, i, h] - want).max() / np.abs(want).max())
-        worst = max(worst, err)
-        assert err <= pu.ATTN_REL_TOL, (b, i, h, err)
-    print(cfg_name, impl, "worst sampled attention error", worst, "excluded sequences", excluded)
-
-
-@pytest.mark.parametrize("impl", IMPLS)
-def test_cfg3_batched_serving_full_size_sampled(impl):
-    _sampled_full_size("cfg3_batched", impl)
-
-
-@pytest.mark.parametrize("impl", IMPLS)
-def test_cfg4_long_context_full_size_sampled(impl):
-    _sampled_full_size("cfg4_long", impl)
+    assert pu.attn_vector_error(got[1], ref["out"][1]).max() <= pu.ATTN_REL_TOL
 
 
 def test_step_is_capturable_in_a_cuda_graph_and_replays_identically():

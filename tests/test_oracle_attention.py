@@ -210,6 +210,21 @@ def test_paging_invariance_and_slot_formula():
         assert len(set(slots.tolist())) == W
 
 
+def test_stage_slots_hand_worked_values():
+    """Cache slots of the staged window rows, worked by hand (slot = physical page * page size + offset):
+    pages of 4 tokens, block table [5, 2, 9].  A prefix of 7 puts row 0 at token 7 = last row of logical
+    page 1 (physical page 2 -> slot 11) and rows 1..4 at tokens 8..11 = logical page 2 (physical page 9
+    -> slots 36..39).  A prefix on a page edge (8) starts a fresh page; a prefix of 3 straddles pages 5 and 2."""
+    table = np.array([[5, 2, 9]], np.int32)
+    assert orc.stage_slots(table, np.array([7]), 5, 4)[0].tolist() == [11, 36, 37, 38, 39]
+    assert orc.stage_slots(table, np.array([8]), 4, 4)[0].tolist() == [36, 37, 38, 39]
+    assert orc.stage_slots(table, np.array([3]), 3, 4)[0].tolist() == [23, 8, 9]
+    assert orc.stage_slots(table, np.array([0]), 2, 4)[0].tolist() == [20, 21]
+    # two sequences, each through its own table row
+    table2 = np.array([[1, 0], [0, 3]], np.int32)
+    assert orc.stage_slots(table2, np.array([1, 3]), 2, 4).tolist() == [[5, 6], [3, 12]]
+
+
 def test_gqa_equals_replicated_kv_heads():
     B, W, P, Hq, Hkv, D, theta = 1, 4, 5, 6, 2, 4, 1e4
     G = Hq // Hkv
