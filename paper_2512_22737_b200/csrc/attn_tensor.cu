@@ -8,7 +8,7 @@
 // rotated K and V were staged there by the RoPE/stage kernel before this kernel starts.
 //
 // One CTA = one (b, g, 128-row tile, key chunk).  Warps 0-3 (128 threads, one query row each) run the
-// online softmax; warp 4 lane 0 issues every MMA; warps 5 and 6 issue the TMA copies of K and V.  Per 64-key tile:
+// online softmax; warp 4 issues every MMA (one elected lane); warps 5 and 6 issue the TMA copies of K and V.  Per 64-key tile:
 //     S[t&1] = Q K_t^T   (tcgen05.mma, 8 k-steps, fp32 in TMEM columns 0..127, double buffered)
 //     softmax threads: tcgen05.ld S row -> mask -> running max (lazy rescale) -> p = 2^(s*c - m*c)
 //                      -> bf16 P tile into shared memory (128-byte swizzle)
@@ -131,10 +131,12 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const uint32_t tmem_O = tmem_base + 128u;     // columns [128,256)
 
   if (warp == 4) {
-    // ------------------------------------------------------------------ MMA issue warp (one lane)
-    // Never waits for an MMA to finish: completion is signalled to the consumers of the result
-    // (S_FULL, O_DONE) and to the producer of the operands (K_FREE, V_FREE) through tcgen05.commit.
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issue warp
+    // All lanes run the loop and wait on the barriers; one elected lane issues (see elect_one()).  The warp
+    // never waits for an MMA to finish: completion is signalled to the consumers of the result (S_FULL,
+    // O_DONE) and to the producer of the operands (K_FREE, V_FREE) through tcgen05.commit.
+    {
+      const bool leader = elect_one();
       bool ok = true;
       const uint32_t idesc_qk = make_idesc(kTileN, false);
       const uint32_t idesc_pv = make_idesc(kD, true);
@@ -145,10 +147,12 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         for (int kk = 0; kk < 8; ++kk) {
           const uint64_t ad = make_desc(sbase + kOffQ + (kk >> 2) * kHalfQ + (kk & 3) * 32u, 16u, 1024u);
           const uint64_t bd = make_desc(sbase + kOffK + st * kStageBytes + (kk >> 2) * kHalfKV + (kk & 3) * 32u, 16u, 1024u);
-          umma(tmem_S + st * 64u, ad, bd, idesc_qk, kk > 0);
+          if (leader) umma(tmem_S + st * 64u, ad, bd, idesc_qk, kk > 0);
         }
-        umma_commit(bar(S_FULL0 + st));
-        umma_commit(bar(K_FREE0 + st));
+        if (leader) {
+          umma_commit(bar(S_FULL0 + st));
+          umma_commit(bar(K_FREE0 + st));
+        }
       };
       ok = mbar_wait(bar(Q_FULL), 0);
       if (ok) ok = mbar_wait(bar(K_FULL0), 0);
@@ -170,12 +174,14 @@ attn_tensor_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         for (int j = 0; j < 4; ++j) {
           const uint64_t ad = make_desc(sbase + kOffP + j * 32u, 16u, 1024u);
           const uint64_t bd = make_desc(sbase + kOffV + st * kStageBytes + j * 2048u, kHalfKV, 1024u);
-          umma(tmem_O, ad, bd, idesc_pv, (t > 0) || (j > 0));
+          if (leader) umma(tmem_O, ad, bd, idesc_pv, (t > 0) || (j > 0));
         }
-        umma_commit(bar(O_DONE));
-        umma_commit(bar(V_FREE0 + st));
+        if (leader) {
+          umma_commit(bar(O_DONE));
+          umma_commit(bar(V_FREE0 + st));
+        }
       }
-      if (!ok) {
+      if (!ok && lane == 0) {
         *abort_flag = 1;
         if (p.status) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
       }

@@ -185,6 +185,32 @@ def test_stale_cache_rows_beyond_the_window_cannot_leak(impl):
     assert pu.attn_vector_error(got, ref["out"]).max() <= pu.ATTN_REL_TOL
 
 
+@pytest.mark.parametrize("where,factor", [(300, 40.0), (0, 40.0), (599, 25.0), (300, 6.0)])
+def test_outlier_keys_move_the_running_maximum_by_large_steps(where, factor):
+    """A cache page scaled up so that its scores lie tens of powers of two above (or below) everything else.
+    With N(0,1) data a row's running maximum creeps up by a bit or two over a whole prefix, so the branch of
+    the tensor path that rescales its accumulator (taken when the maximum grows by more than 2^8) never runs;
+    here it runs in the middle of the prefix, right after the first tile, and on the last tile.  Scores that
+    large multiply the effect of the bf16 rounding of the rotated q by the same factor, so the fp64 oracle is
+    not the right yardstick; the CUDA-core path is: it reads the same rounded q and the same cache, computes
+    the softmax in fp32 and rescales on every page."""
+    import parity_util as pu
+    from workloads import bf16_bits, bf16_to_f32
+    cfg = _small_qwen(batch=2, window=16, prefix_lo=600, prefix_hi=600, vocab=1024, name="outlier")
+    inp = make_step(cfg, seed=int(where + factor))
+    for b in range(2):
+        pg = inp["block_table"][b, (where + 16 * b) // 16]
+        page = bf16_to_f32(inp["k_cache"][pg].reshape(-1)) * np.float32(factor)
+        inp["k_cache"][pg] = bf16_bits(page).reshape(inp["k_cache"][pg].shape)
+    outs = {}
+    for impl in IMPLS:
+        step, _ = pu.run_gpu_step(cfg, inp, attn_impl=impl)
+        assert int(step.status.item()) == 0
+        outs[impl] = pu.bf16_from_device(step.out)
+        assert np.isfinite(outs[impl]).all()
+    assert pu.attn_vector_error(outs["tensor"], outs["generic"]).max() <= pu.ATTN_REL_TOL
+
+
 def test_tensor_path_refuses_shapes_it_does_not_cover():
     import paper_2512_22737_b200 as w
     cfg = w.make_config(batch=1, window=8, n_q_heads=4, n_kv_heads=2, head_dim=64, max_pages_per_seq=8,
