@@ -211,6 +211,8 @@ size_t wedlm_confidence_workspace_bytes(const wedlm_config_t* cfg);
  *   committed_tokens out i32 [B,W] first committed_count[b] entries valid, rest -1
  *   committed_count  out i32 [B]
  *   filled_count     out i32 [B]  masks filled this step
+ *   status        in/out i32 [1] or NULL; WEDLM_STATUS_WAIT_EXPIRED is OR-ed in if a bounded on-chip wait of the
+ *                               streaming pass gave up (the statistics of some rows are then missing)
  * Order of operations per sequence: commit the n_commit leading slots; among the remaining
  * masks compute d = logical distance to the leftmost mask; select; if nothing is selected and a
  * mask exists, select the single best-scoring mask (leftmost on ties) so that decoding always
@@ -238,7 +240,7 @@ int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const
                             int32_t* argmax, float* maxprob, float* entropy, float* lse,
                             int32_t* committed_tokens, int32_t* committed_count,
                             int32_t* filled_count, void* workspace, size_t workspace_bytes,
-                            void* stream);
+                            int32_t* status, void* stream);
 
 /*
  * wedlm_confidence_commit fused with the LM head (Algorithm 1 takes its logits from Forward; here the last
@@ -264,7 +266,7 @@ int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, co
                                    int32_t* argmax, float* maxprob, float* entropy, float* lse,
                                    int32_t* committed_tokens, int32_t* committed_count,
                                    int32_t* filled_count, void* workspace, size_t workspace_bytes,
-                                   void* stream);
+                                   int32_t* status, void* stream);
 
 /*
  * wedlm_confidence_commit without a workspace argument, for hosts that must not allocate device
@@ -297,7 +299,7 @@ int wedlm_confidence_commit_static(const wedlm_config_t* cfg, const void* logits
                                    int32_t* window_len, int32_t* remaining_budget,
                                    int32_t* argmax, float* maxprob, float* entropy, float* lse,
                                    int32_t* committed_tokens, int32_t* committed_count,
-                                   int32_t* filled_count, void* stream);
+                                   int32_t* filled_count, int32_t* status, void* stream);
 
 /*
  * Commit + shift + Refill of Algorithm 1 alone, for callers that did the selection themselves

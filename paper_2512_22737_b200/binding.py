@@ -89,16 +89,16 @@ def load_library() -> ctypes.CDLL:
     lib.wedlm_confidence_commit.restype = ctypes.c_int
     lib.wedlm_confidence_commit.argtypes = [cfgp, vp, i32p, i32p, i32p, i32p, u8p, i32p, i32p, i32p,
                                             i32p, f32p, f32p, f32p, i32p, i32p, i32p, vp,
-                                            ctypes.c_size_t, vp]
+                                            ctypes.c_size_t, i32p, vp]
     lib.wedlm_confidence_commit_static.restype = ctypes.c_int
     lib.wedlm_confidence_commit_static.argtypes = [cfgp, vp, i32p, i32p, i32p, i32p, u8p, i32p, i32p, i32p,
-                                                   i32p, f32p, f32p, f32p, i32p, i32p, i32p, vp]
+                                                   i32p, f32p, f32p, f32p, i32p, i32p, i32p, i32p, vp]
     lib.wedlm_lmhead_confidence_workspace_bytes.restype = ctypes.c_size_t
     lib.wedlm_lmhead_confidence_workspace_bytes.argtypes = [cfgp]
     lib.wedlm_lmhead_confidence_commit.restype = ctypes.c_int
     lib.wedlm_lmhead_confidence_commit.argtypes = [cfgp, ctypes.c_int32, vp, vp, i32p, ctypes.c_float, i32p, i32p, i32p,
                                                    i32p, u8p, i32p, i32p, i32p, i32p, f32p, f32p, f32p, i32p, i32p,
-                                                   i32p, vp, ctypes.c_size_t, vp]
+                                                   i32p, vp, ctypes.c_size_t, i32p, vp]
     lib.wedlm_window_refill.restype = ctypes.c_int
     lib.wedlm_window_refill.argtypes = [cfgp, i32p, i32p, u8p, i32p, i32p, i32p, i32p, i32p, vp]
     lib.wedlm_step_host_workspace_bytes.restype = ctypes.c_size_t
@@ -232,7 +232,7 @@ def wedlm_confidence_workspace_bytes(cfg) -> int:
 
 def wedlm_confidence_commit(cfg, logits, perm, n_filled, n_commit, window_tokens, filled, prefix_len,
                             window_len, remaining_budget, argmax, maxprob, entropy, lse,
-                            committed_tokens, committed_count, filled_count, workspace, stream=None) -> None:
+                            committed_tokens, committed_count, filled_count, workspace, status=None, stream=None) -> None:
     i32, u8, f32 = torch.int32, torch.uint8, torch.float32
     _check(load_library().wedlm_confidence_commit(
         ctypes.byref(cfg), _ptr(logits, cfg.torch_dtype, "logits"), _ptr(perm, i32, "perm"),
@@ -243,7 +243,7 @@ def wedlm_confidence_commit(cfg, logits, perm, n_filled, n_commit, window_tokens
         _ptr(lse, f32, "lse"), _ptr(committed_tokens, i32, "committed_tokens"),
         _ptr(committed_count, i32, "committed_count"), _ptr(filled_count, i32, "filled_count"),
         _ptr(workspace, None, "workspace"), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
-        _stream(stream)), "wedlm_confidence_commit")
+        _ptr(status, i32, "status"), _stream(stream)), "wedlm_confidence_commit")
 
 
 def wedlm_lmhead_confidence_workspace_bytes(cfg) -> int:
@@ -252,7 +252,7 @@ def wedlm_lmhead_confidence_workspace_bytes(cfg) -> int:
 
 def wedlm_lmhead_confidence_commit(cfg, hidden_states, lm_head, tilt_ids, tilt, perm, n_filled, n_commit, window_tokens,
                                    filled, prefix_len, window_len, remaining_budget, argmax, maxprob, entropy, lse,
-                                   committed_tokens, committed_count, filled_count, workspace, stream=None) -> None:
+                                   committed_tokens, committed_count, filled_count, workspace, status=None, stream=None) -> None:
     """Confidence/commit straight from the hidden states [B,W,H] and the output embedding [V,H] (bf16)."""
     i32, u8, f32, bf = torch.int32, torch.uint8, torch.float32, torch.bfloat16
     _check(load_library().wedlm_lmhead_confidence_commit(
@@ -264,7 +264,7 @@ def wedlm_lmhead_confidence_commit(cfg, hidden_states, lm_head, tilt_ids, tilt, 
         _ptr(entropy, f32, "entropy"), _ptr(lse, f32, "lse"), _ptr(committed_tokens, i32, "committed_tokens"),
         _ptr(committed_count, i32, "committed_count"), _ptr(filled_count, i32, "filled_count"),
         _ptr(workspace, None, "workspace"), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
-        _stream(stream)), "wedlm_lmhead_confidence_commit")
+        _ptr(status, i32, "status"), _stream(stream)), "wedlm_lmhead_confidence_commit")
 
 
 WEDLM_STATIC_SCRATCH_BYTES = 4 << 20
@@ -273,7 +273,7 @@ WEDLM_ERR_STATIC_SCRATCH = -6
 
 def wedlm_confidence_commit_static(cfg, logits, perm, n_filled, n_commit, window_tokens, filled, prefix_len,
                                    window_len, remaining_budget, argmax, maxprob, entropy, lse,
-                                   committed_tokens, committed_count, filled_count, stream=None) -> None:
+                                   committed_tokens, committed_count, filled_count, status=None, stream=None) -> None:
     """wedlm_confidence_commit for callers that may not allocate device memory (a process whose HBM is
     already committed to a cache pool, a loop that bans allocator calls): same inputs and outputs, no
     workspace; the scratch is a fixed 4 MiB array inside the library.  Raises WedlmError with code
@@ -288,7 +288,7 @@ def wedlm_confidence_commit_static(cfg, logits, perm, n_filled, n_commit, window
         _ptr(argmax, i32, "argmax"), _ptr(maxprob, f32, "maxprob"), _ptr(entropy, f32, "entropy"),
         _ptr(lse, f32, "lse"), _ptr(committed_tokens, i32, "committed_tokens"),
         _ptr(committed_count, i32, "committed_count"), _ptr(filled_count, i32, "filled_count"),
-        _stream(stream)), "wedlm_confidence_commit_static")
+        _ptr(status, i32, "status"), _stream(stream)), "wedlm_confidence_commit_static")
 
 
 def wedlm_window_refill(cfg, n_commit, window_tokens, filled, prefix_len, window_len, remaining_budget,
@@ -411,7 +411,7 @@ class DecodeStep:
         wedlm_confidence_commit(self.cfg, logits, self.perm, self.n_filled, self.n_commit, window_tokens, filled,
                                 prefix_len, window_len, remaining_budget, self.argmax, self.maxprob, self.entropy,
                                 self.lse, self.committed_tokens, self.committed_count, self.filled_count,
-                                self.conf_ws)
+                                self.conf_ws, self.status)
 
     def capture_graph(self, d: Dict[str, torch.Tensor], window_len=None, remaining_budget=None) -> "torch.cuda.CUDAGraph":
         """Capture reorder -> attention -> confidence/commit on these fixed buffers into a CUDA graph.

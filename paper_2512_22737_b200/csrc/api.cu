@@ -249,7 +249,7 @@ int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const
                             uint8_t* filled, int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
                             int32_t* argmax, float* maxprob, float* entropy, float* lse, int32_t* committed_tokens,
                             int32_t* committed_count, int32_t* filled_count, void* workspace, size_t workspace_bytes,
-                            void* stream) {
+                            int32_t* status, void* stream) {
   int rc = check_config(cfg, false, true);
   if (rc != WEDLM_OK) return rc;
   if (cfg->batch == 0) return WEDLM_OK;
@@ -259,7 +259,7 @@ int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const
   if (workspace_bytes < confidence_workspace_bytes(cfg)) return WEDLM_ERR_WORKSPACE_TOO_SMALL;
   return launch_confidence(make_shape(cfg), cfg, logits, perm, n_filled, n_commit, window_tokens, filled, prefix_len,
                            window_len, remaining_budget, argmax, maxprob, entropy, lse, committed_tokens,
-                           committed_count, filled_count, workspace, (cudaStream_t)stream);
+                           committed_count, filled_count, workspace, status, (cudaStream_t)stream);
 }
 
 size_t wedlm_lmhead_confidence_workspace_bytes(const wedlm_config_t* cfg) {
@@ -274,7 +274,7 @@ int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, co
                                    uint8_t* filled, int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
                                    int32_t* argmax, float* maxprob, float* entropy, float* lse, int32_t* committed_tokens,
                                    int32_t* committed_count, int32_t* filled_count, void* workspace, size_t workspace_bytes,
-                                   void* stream) {
+                                   int32_t* status, void* stream) {
   int rc = check_config(cfg, false, true);
   if (rc != WEDLM_OK) return rc;
   if (cfg->dtype != WEDLM_DTYPE_BF16 || hidden < 64 || hidden % 64 != 0) return WEDLM_ERR_UNSUPPORTED;
@@ -288,7 +288,7 @@ int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, co
   Shape s = make_shape(cfg);
   cudaStream_t st = (cudaStream_t)stream;
   int n_tiles = 0;
-  rc = launch_lmhead_conf(s, hidden, hidden_states, lm_head, tilt_ids, tilt, n_filled, window_len, workspace, &n_tiles, st);
+  rc = launch_lmhead_conf(s, hidden, hidden_states, lm_head, tilt_ids, tilt, n_filled, window_len, workspace, &n_tiles, status, st);
   if (rc != WEDLM_OK) return rc;
   return launch_conf_commit(s, cfg, n_tiles, workspace, perm, n_filled, n_commit, window_tokens, filled,
                             prefix_len, window_len, remaining_budget, argmax, maxprob, entropy, lse, committed_tokens,
@@ -506,7 +506,7 @@ int wedlm_step_host(const wedlm_config_t* cfg, uint8_t* h_filled, int32_t* h_win
                                reinterpret_cast<float*>(ws + p.off_maxprob), reinterpret_cast<float*>(ws + p.off_entropy),
                                reinterpret_cast<float*>(ws + p.off_lse), reinterpret_cast<int32_t*>(ws + p.off_ctok),
                                reinterpret_cast<int32_t*>(ws + p.off_ccount), reinterpret_cast<int32_t*>(ws + p.off_fcount),
-                               ws + p.off_conf_ws, p.conf_ws_bytes, stream);
+                               ws + p.off_conf_ws, p.conf_ws_bytes, status, stream);
   if (rc != WEDLM_OK) return rc;
   ok = down(h_committed_tokens, p.off_ctok, B * W * 4) && down(h_committed_count, p.off_ccount, B * 4) &&
        down(h_filled, p.off_filled, B * W) && down(h_window_tokens, p.off_tokens, B * W * 4) &&

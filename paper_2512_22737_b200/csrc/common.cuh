@@ -98,7 +98,7 @@ int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* log
                       const int32_t* n_filled, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
                       int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget, int32_t* argmax,
                       float* maxprob, float* entropy, float* lse, int32_t* committed_tokens,
-                      int32_t* committed_count, int32_t* filled_count, void* workspace, cudaStream_t st);
+                      int32_t* committed_count, int32_t* filled_count, void* workspace, int32_t* status, cudaStream_t st);
 
 int launch_conf_commit(const Shape& s, const wedlm_config_t* cfg, int n_chunks, const void* partials, const int32_t* perm,
                        const int32_t* n_filled, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
@@ -110,7 +110,7 @@ int launch_conf_commit(const Shape& s, const wedlm_config_t* cfg, int n_chunks, 
 int lmhead_conf_tiles(int vocab);
 int launch_lmhead_conf(const Shape& s, int hidden, const void* hidden_states, const void* lm_head, const int32_t* tilt_ids,
                        float tilt, const int32_t* n_filled, const int32_t* window_len, void* partials, int* n_tiles_out,
-                       cudaStream_t st);
+                       int32_t* status, cudaStream_t st);
 
 // Dual-Stream Masking (training forward): input construction and the per-unit page tables.
 int launch_dual_stream_construct(int N, int L, int B, int K, int mask_id, const int32_t* tokens, const uint8_t* masked,

@@ -220,7 +220,7 @@ __device__ __forceinline__ void cs_consumer_sync() {     // the consumer threads
 __global__ void __launch_bounds__(kStreamThreads + 32)
 conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv_bfloat16* __restrict__ logits,
                    const int32_t* __restrict__ n_filled, const int32_t* __restrict__ window_len,
-                   float4* __restrict__ part) {
+                   float4* __restrict__ part, int32_t* status) {
   extern __shared__ __align__(128) unsigned char cs_smem[];
   unsigned char* stage_mem = cs_smem;                                       // kStreamStages x 16 KB
   uint64_t* full = reinterpret_cast<uint64_t*>(cs_smem + kStreamStages * kStreamChunk * 2);
@@ -230,7 +230,9 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
   __shared__ float fs[kStreamThreads / 32];
   __shared__ float ft[kStreamThreads / 32];
   __shared__ int fa;
+  __shared__ volatile int gave_up;                   // a bounded wait expired: every consumer leaves at the next barrier
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) gave_up = 0;
   long long cursor = blockIdx.x;                     // next candidate item of this block (producer only)
 
   // producer: put the next active item of this block into stage st, or -1 when the block is done;
@@ -277,7 +279,10 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
       bool more = true;
       for (uint32_t n = 0; more; ++n) {
         const int st = n & (kStreamStages - 1);
-        if (n >= kStreamStages && !cs_mbar_wait(cs_smem_u32(empty + st), ((n / kStreamStages) - 1) & 1u)) break;
+        if (n >= kStreamStages && !cs_mbar_wait(cs_smem_u32(empty + st), ((n / kStreamStages) - 1) & 1u)) {
+          if (status) atomicOr(status, WEDLM_STATUS_WAIT_EXPIRED);
+          break;
+        }
         more = produce(st);
       }
     }
@@ -286,9 +291,12 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
 
   for (uint32_t n = 0;; ++n) {
     const int st = n & (kStreamStages - 1);
-    if (!cs_mbar_wait(cs_smem_u32(full + st), (n / kStreamStages) & 1u)) return;   // bounded; never expected
-    const int row = item_of[st].x, chunk = item_of[st].y;
-    if (row < 0) break;
+    // Bounded, never expected to expire.  A thread whose wait does expire must not leave by itself (the others
+    // would wait for it at the block barrier below for ever): it raises a flag and carries on to that barrier,
+    // behind which all consumers leave together.
+    if (!cs_mbar_wait(cs_smem_u32(full + st), (n / kStreamStages) & 1u)) gave_up = 1;
+    const int row = gave_up ? 0 : item_of[st].x, chunk = gave_up ? 0 : item_of[st].y;
+    if (row < 0) break;                              // end marker: seen by all consumers alike (set before the barrier's arrival)
     const int base = chunk * kStreamChunk;
     const uint4* src = reinterpret_cast<const uint4*>(stage_mem + (size_t)st * kStreamChunk * 2);
     uint32_t w[kStreamVecs * 4];
@@ -324,6 +332,10 @@ conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv
     if (lane == 0) fm[warp] = m;
     if (tid == 0) fa = 0x7fffffff;
     cs_consumer_sync();                              // also: every consumer holds its part of stage st in registers
+    if (gave_up) {
+      if (tid == 0 && status) atomicOr(status, WEDLM_STATUS_WAIT_EXPIRED);
+      return;
+    }
     if (tid == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(cs_smem_u32(empty + st)) : "memory");
     m = fm[0];
 #pragma unroll
@@ -711,7 +723,7 @@ int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* log
                       const int32_t* n_filled, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
                       int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget, int32_t* argmax,
                       float* maxprob, float* entropy, float* lse, int32_t* committed_tokens,
-                      int32_t* committed_count, int32_t* filled_count, void* workspace, cudaStream_t st) {
+                      int32_t* committed_count, int32_t* filled_count, void* workspace, int32_t* status, cudaStream_t st) {
   const int n_chunks = conf_chunks(cfg);
   const long long blocks = (long long)s.B * s.W * n_chunks;
   if (blocks > 0x7fffffffLL) return WEDLM_ERR_UNSUPPORTED;
@@ -732,7 +744,7 @@ int launch_confidence(const Shape& s, const wedlm_config_t* cfg, const void* log
       long long grid = (long long)device_sm_count() * kStreamBlocksPerSM;
       if (grid > blocks) grid = blocks;
       conf_stream_kernel<<<(unsigned)grid, kStreamThreads + 32, smem, st>>>(s.W, s.V, n_chunks, blocks, (const T*)logits, n_filled,
-                                                                      window_len, part);
+                                                                      window_len, part, status);
     } else {
       conf_partial_kernel<T, false><<<(unsigned)blocks, kConfThreads, 0, st>>>(s.W, s.V, n_chunks, (const T*)logits, n_filled, window_len, part);
     }
@@ -851,7 +863,7 @@ extern "C" int wedlm_confidence_commit_static(const wedlm_config_t* cfg, const v
                                               int32_t* window_len, int32_t* remaining_budget, int32_t* argmax,
                                               float* maxprob, float* entropy, float* lse,
                                               int32_t* committed_tokens, int32_t* committed_count,
-                                              int32_t* filled_count, void* stream) {
+                                              int32_t* filled_count, int32_t* status, void* stream) {
   const size_t need = wedlm_confidence_workspace_bytes(cfg);     // 0 for a NULL / invalid config
   if (need == 0) return WEDLM_ERR_INVALID_ARG;
   if (need > (size_t)WEDLM_STATIC_SCRATCH_BYTES) return WEDLM_ERR_STATIC_SCRATCH;
@@ -862,5 +874,5 @@ extern "C" int wedlm_confidence_commit_static(const wedlm_config_t* cfg, const v
   // has to start at zero and the previous call's contents are harmless.
   return wedlm_confidence_commit(cfg, logits, perm, n_filled, n_commit, window_tokens, filled, prefix_len, window_len,
                                  remaining_budget, argmax, maxprob, entropy, lse, committed_tokens, committed_count,
-                                 filled_count, scratch, (size_t)WEDLM_STATIC_SCRATCH_BYTES, stream);
+                                 filled_count, scratch, (size_t)WEDLM_STATIC_SCRATCH_BYTES, status, stream);
 }

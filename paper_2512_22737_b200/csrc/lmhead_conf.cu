@@ -9,7 +9,7 @@
 // accumulators of 256 TMEM columns each), so the output embedding is streamed from HBM once when
 // B*W <= 256.  One persistent CTA per SM walks the items.  Warp 9 feeds a 3-stage ring with TMA (hidden
 // states 2 x [128 x 64], embedding [tile_n x 64] per stage, 128-byte swizzle), warp 8 issues tcgen05.mma
-// (128 x tile_n x 16, 8 per stage) and releases stages through tcgen05.commit, warps 0-7 read their row of
+// (128 x tile_n x 16, 8 per stage; one elected lane, the whole warp runs the loop) and releases stages through tcgen05.commit, warps 0-7 read their row of
 // the accumulators back with tcgen05.ld and reduce it.  The wide tile matters: every item re-reads the
 // hidden states from L2, and that traffic, not HBM, bounds the kernel.  All waits are bounded.
 #include <cuda.h>
@@ -46,6 +46,7 @@ struct LmParams {
   const int32_t* n_filled;
   const int32_t* window_len;
   float4* part;
+  int32_t* status;
 };
 
 // Persistent CTAs: work item = (row chunk, vocabulary tile), items strided over the grid.
@@ -94,10 +95,13 @@ lmhead_conf_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
           tma_load_2d(sbase + kLmOffB + st * kLmStrideB, &tm_w, k * kLmTileK, n0, bar(LM_FULL0 + st));
         }
       }
+      if (!ok && p.status) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
     }
   } else if (warp == 8) {
-    // ------------------------------------------------------------------ MMA issue (one lane)
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issue
+    // all lanes run the loop and wait on the barriers, one elected lane issues (see elect_one())
+    {
+      const bool leader = elect_one();
       const uint32_t idesc = make_idesc(p.tile_n, false);
       uint32_t kq = 0, it = 0;
       bool ok = true;
@@ -118,13 +122,14 @@ lmhead_conf_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
             for (int kk = 0; kk < 4; ++kk) {
               const uint64_t ad = make_desc(sbase + kLmOffA + (st * 2 + mt) * kLmBytesA + kk * 32u, 16u, 1024u);
               const uint64_t bd = make_desc(sbase + kLmOffB + st * kLmStrideB + kk * 32u, 16u, 1024u);
-              umma(tmem_base + (uint32_t)mt * 256u, ad, bd, idesc, (k > 0) || (kk > 0));
+              if (leader) umma(tmem_base + (uint32_t)mt * 256u, ad, bd, idesc, (k > 0) || (kk > 0));
             }
           }
-          umma_commit(bar(LM_FREE0 + st));
+          if (leader) umma_commit(bar(LM_FREE0 + st));
         }
-        umma_commit(bar(LM_ACC_FULL));            // arrives when every MMA of this item has completed
+        if (leader) umma_commit(bar(LM_ACC_FULL));            // arrives when every MMA of this item has completed
       }
+      if (!ok && lane == 0 && p.status) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
     }
   } else {
     // ------------------------------------------------------------------ reduction warps: one row per thread
@@ -142,7 +147,10 @@ lmhead_conf_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         active = i >= p.n_filled[b] && i < L;
       }
       const int tilt_col = (active && p.tilt_ids) ? p.tilt_ids[row] - n0 : -1;     // column of this tile, if any
-      if (!mbar_wait(bar(LM_ACC_FULL), it & 1u)) break;
+      if (!mbar_wait(bar(LM_ACC_FULL), it & 1u)) {
+        if (p.status && (tid & 127) == 0) atomicOr(p.status, WEDLM_STATUS_WAIT_EXPIRED);
+        break;
+      }
       tc_fence_after();
       if (mt < n_mt) {
         const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)mt * 256u;
@@ -186,8 +194,12 @@ lmhead_conf_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
             t = fmaf(d, ex, t);
           }
         }
-        if (active && m > -CUDART_INF_F)
-          p.part[(size_t)row * p.n_tiles + tile] = make_float4(m, s, t * 0.6931471805599453f, __int_as_float(a));
+        // every active row gets a partial for every tile: a tile without a finite logit leaves an empty one, which
+        // the merge skips (the workspace is not cleared between calls)
+        if (active)
+          p.part[(size_t)row * p.n_tiles + tile] = (m > -CUDART_INF_F)
+              ? make_float4(m, s, t * 0.6931471805599453f, __int_as_float(a))
+              : make_float4(-CUDART_INF_F, 0.f, 0.f, __int_as_float(0x7fffffff));
       }
       tc_fence_before();
       mbar_arrive(bar(LM_ACC_FREE));               // this thread no longer needs the accumulators
@@ -235,7 +247,7 @@ int lmhead_conf_tiles(int vocab) { return (vocab + 127) / 128; }
 
 int launch_lmhead_conf(const Shape& s, int hidden, const void* hidden_states, const void* lm_head, const int32_t* tilt_ids,
                        float tilt, const int32_t* n_filled, const int32_t* window_len, void* partials, int* n_tiles_out,
-                       cudaStream_t st) {
+                       int32_t* status, cudaStream_t st) {
   auto encode = lm_get_encode();
   if (!encode) return WEDLM_ERR_CUDA;
   const int R = s.B * s.W;
@@ -269,6 +281,7 @@ int launch_lmhead_conf(const Shape& s, int hidden, const void* hidden_states, co
   p.n_row_chunks = row_chunks;
   p.tilt = tilt; p.tilt_ids = tilt_ids; p.n_filled = n_filled; p.window_len = window_len;
   p.part = reinterpret_cast<float4*>(partials);
+  p.status = status;
   const int n_items = p.n_tiles * p.n_row_chunks;
   const int grid = n_items < sms ? n_items : sms;       // one persistent CTA per SM (the whole tensor memory each)
   lmhead_conf_kernel<<<grid, kLmThreads, kLmSmem, st>>>(tm_h, tm_w, p);

@@ -40,8 +40,9 @@ def _case(B, W, V, H, seed, boost=6.0, window_len=None, budget=None, commit_mode
     w.wedlm_lmhead_confidence_commit(c, w.to_device(hid), w.to_device(emb), w.to_device(tilt_ids), boost, step.perm,
                                      step.n_filled, step.n_commit, d["window_tokens"], d["filled"], d["prefix_len"], wl, bud,
                                      step.argmax, step.maxprob, step.entropy, step.lse, step.committed_tokens,
-                                     step.committed_count, step.filled_count, ws)
+                                     step.committed_count, step.filled_count, ws, step.status)
     torch.cuda.synchronize()
+    assert int(step.status.item()) == 0
     d["window_len"], d["remaining_budget"] = wl, bud
     # arg-max: exact unless the two best logits of the row are within the 1e-3 band
     am = step.argmax.cpu().numpy()
