@@ -104,10 +104,12 @@ class ClockSampler:
         if self.ok and self.thread.is_alive():
             self.thread.join(timeout=2)
 
-    def summary(self):
+    def summary(self, tag="timed"):
+        """Median SM clock and the union of throttle reasons over the samples taken while `tag` was set
+        (the headline line uses the samples inside the timed region of the main workload)."""
         if not self.ok or not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
-        timed = [s for s in self.samples if s[3] == "timed"]
+        timed = [s for s in self.samples if s[3] == tag]
         use = timed if len(timed) >= 3 else [s for s in self.samples if s[3] != "idle"]
         if not use:
             use = self.samples
@@ -115,8 +117,9 @@ class ClockSampler:
         for s in use:
             mask |= s[2]
         reasons = [name for bit, name in self.REASONS.items() if mask & bit]
-        return {"sm_mhz": statistics.median(s[1] for s in use), "sm_max_mhz": self.max_mhz,
-                "reasons": reasons, "samples": len(use), "samples_in_timed_region": len(timed)}
+        return {"sm_mhz": statistics.median(s[1] for s in use), "sm_min_mhz": min(s[1] for s in use),
+                "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(use),
+                "samples_in_timed_region": len(timed)}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -131,7 +134,12 @@ def algorithmic_bytes(cfg, inp):
     q_io = 2 * B * W * cfg.n_q_heads * cfg.head_dim * elem                # rotated q read + out write
     n_mask_rows = int((inp["filled"] == 0).sum())
     logits = n_mask_rows * cfg.vocab * elem
-    return {"attn_kernel": kv + q_io, "kv_stream": kv, "logits_stream": logits, "mask_rows": n_mask_rows}
+    # attention flops: QK^T and PV, 2 D flops per (row, key, query head) each; row i of sequence b sees P_b + i + 1 keys
+    keys = int((inp["prefix_len"].astype(np.int64) * W + W * (W + 1) // 2).sum())
+    flops = 4.0 * cfg.head_dim * cfg.n_q_heads * keys
+    prefix_only = int(inp["prefix_len"].astype(np.int64).sum()) * cfg.n_kv_heads * cfg.head_dim * 2 * elem
+    return {"attn_kernel": kv + q_io, "kv_stream": kv, "kv_prefix_only": prefix_only, "logits_stream": logits,
+            "mask_rows": n_mask_rows, "attn_flops": flops}
 
 
 def slice_batch(inp, n):
@@ -250,8 +258,12 @@ class Workload:
         s.confidence_commit(d["logits"], d["window_tokens"], d["filled"], d["prefix_len"])
 
 
-def time_workload(wl, steps, warmup, sampler=None, tag="timed"):
-    """warmup + `steps` timed iterations; returns (ms_per_step, attn_kernel_ms_avg, committed, launches)."""
+def time_workload(wl, steps, warmup, sampler=None, tag="timed", min_region_s=1.0, max_blocks=2000):
+    """`warmup` untimed steps, then blocks of exactly `steps` steps, each block bracketed by CUDA events on the
+    launching stream, repeated back to back until the timed blocks add up to `min_region_s` (steady state: the
+    clocks have settled under the load).  The window state is restored between blocks, outside the events.
+    Returns a dict: mean / median / best ms per step over the blocks, the mean duration of the attention kernel
+    (events placed inside wedlm_window_attn around that kernel), commits per step, launches per step."""
     import torch
     import paper_2512_22737_b200 as w
     wl.reset_states()
@@ -265,23 +277,30 @@ def time_workload(wl, steps, warmup, sampler=None, tag="timed"):
         b.record()
     torch.cuda.synchronize()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    l0 = w.wedlm_launch_count()
+    block_ms, attn_ms_sum, launches = [], 0.0, 0
     if sampler:
         sampler.tag = tag
-    start.record()
-    for i in range(steps):
-        wl.run_step(profile_events=evs[i])
-    stop.record()
-    torch.cuda.synchronize()
+    while sum(block_ms) < min_region_s * 1e3 and len(block_ms) < max_blocks:
+        wl.reset_states()
+        l0 = w.wedlm_launch_count()
+        start.record()
+        for i in range(steps):
+            wl.run_step(profile_events=evs[i])
+        stop.record()
+        torch.cuda.synchronize()
+        launches = w.wedlm_launch_count() - l0
+        block_ms.append(start.elapsed_time(stop))
+        attn_ms_sum += sum(a.elapsed_time(b) for a, b in evs)
     if sampler:
         sampler.tag = "other"
-    launches = w.wedlm_launch_count() - l0
-    ms = start.elapsed_time(stop) / steps
-    attn_ms = sum(a.elapsed_time(b) for a, b in evs) / steps
-    return ms, attn_ms, committed, launches
+    n_blocks = len(block_ms)
+    per_step = sorted(x / steps for x in block_ms)
+    return {"ms": sum(block_ms) / (n_blocks * steps), "ms_median": statistics.median(per_step), "ms_best": per_step[0],
+            "attn_ms": attn_ms_sum / (n_blocks * steps), "committed": committed, "launches": launches,
+            "blocks": n_blocks, "region_s": sum(block_ms) * 1e-3}
 
 
-def time_graph(wl, steps, warmup):
+def time_graph(wl, steps, warmup, min_region_s=0.25):
     """The same step captured once into a CUDA graph (the window state is restored from pristine copies
     inside the graph, three small device copies) and replayed: launch overhead removed.  Uses the first
     copy of the large streams, so workloads that fit in L2 run warm here."""
@@ -308,23 +327,31 @@ def time_graph(wl, steps, warmup):
         graph.replay()
     torch.cuda.synchronize()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    start.record()
-    for _ in range(steps):
-        graph.replay()
-    stop.record()
-    torch.cuda.synchronize()
-    return start.elapsed_time(stop) / steps
+    total, n = 0.0, 0
+    while total < min_region_s * 1e3 and n < 2000 * steps:
+        start.record()
+        for _ in range(steps):
+            graph.replay()
+        stop.record()
+        torch.cuda.synchronize()
+        total += start.elapsed_time(stop)
+        n += steps
+    return total / n
 
 
-def time_e2e(wl, steps, warmup, sampler=None):
-    """The same step through wedlm_step_host, the library's call for step inputs that live in HOST memory:
-    every iteration sends the window state, block table, q/k/v and the logits rows the step reads from
-    page-locked host buffers, runs the three calls and brings the commit results and the new window state
-    back.  The KV cache is resident device state, as in a serving engine."""
+def time_e2e(wl, steps, warmup, sampler=None, mode="lmhead", hidden=4096, lm_head=None):
+    """The same step through the library's calls for step inputs that live in HOST memory: every iteration sends
+    the window state, block table and q/k/v from page-locked host buffers, runs reorder -> attention ->
+    confidence/commit and brings the commit results and the new window state back.  The KV cache is resident
+    device state, as in a serving engine.
+      mode "lmhead": wedlm_step_host_lmhead - the hidden states of the window rows come from the host, the output
+                     embedding is resident and the LM head runs inside the step (what a serving loop hands over);
+      mode "logits": wedlm_step_host - the [B,W,V] logits themselves come from the host (only the rows the step
+                     reads are sent); this leg measures the host link."""
     import torch
     import paper_2512_22737_b200 as w
     inp = wl.inp
-    names = ["filled", "window_tokens", "prefix_len", "block_table", "q", "k", "v", "logits"]
+    names = ["filled", "window_tokens", "prefix_len", "block_table", "q", "k", "v"] + (["logits"] if mode == "logits" else [])
     src = {}
     for k in names:
         a = inp[k]
@@ -335,26 +362,41 @@ def time_e2e(wl, steps, warmup, sampler=None):
     ct = torch.empty(B, W, dtype=torch.int32).pin_memory()
     cc = torch.empty(B, dtype=torch.int32).pin_memory()
     fc = torch.empty(B, dtype=torch.int32).pin_memory()
-    ws = torch.empty(w.wedlm_step_host_workspace_bytes(wl.c), dtype=torch.uint8, device="cuda")
     big = wl.big[0]
     elem = 2 if wl.cfg.dtype == "bf16" else 4
     n_mask_rows = int((inp["filled"] == 0).sum())
-    h2d = sum(host[k].numel() * host[k].element_size() for k in names if k != "logits") + n_mask_rows * wl.cfg.vocab * elem
+    small = sum(host[k].numel() * host[k].element_size() for k in names if k != "logits")
     d2h = sum(t.numel() * t.element_size() for t in (ct, cc, fc)) + sum(host[k].numel() * host[k].element_size() for k in state)
+    if mode == "logits":
+        ws = torch.empty(w.wedlm_step_host_workspace_bytes(wl.c), dtype=torch.uint8, device="cuda")
+        h2d = small + n_mask_rows * wl.cfg.vocab * elem
+
+        def call():
+            w.wedlm_step_host(wl.c, host["filled"], host["window_tokens"], host["prefix_len"], None, None, host["block_table"],
+                              host["q"], host["k"], host["v"], host["logits"], big["k_cache"], big["v_cache"], ct, cc, fc, ws,
+                              wl.step.status)
+    else:
+        g = torch.Generator().manual_seed(251222737)
+        h_hid = torch.randn(B, W, hidden, generator=g).to(torch.bfloat16).pin_memory()
+        ws = torch.empty(w.wedlm_step_host_lmhead_workspace_bytes(wl.c, hidden), dtype=torch.uint8, device="cuda")
+        h2d = small + h_hid.numel() * 2
+
+        def call():
+            w.wedlm_step_host_lmhead(wl.c, host["filled"], host["window_tokens"], host["prefix_len"], None, None,
+                                     host["block_table"], host["q"], host["k"], host["v"], h_hid, lm_head, None, 0.0,
+                                     big["k_cache"], big["v_cache"], ct, cc, fc, ws, wl.step.status)
 
     def one():
         for k in state:                       # the step updates the window state in place: start from the same one
             host[k].copy_(src[k])
-        w.wedlm_step_host(wl.c, host["filled"], host["window_tokens"], host["prefix_len"], None, None, host["block_table"],
-                          host["q"], host["k"], host["v"], host["logits"], big["k_cache"], big["v_cache"], ct, cc, fc, ws,
-                          wl.step.status)
+        call()
         torch.cuda.synchronize()              # the caller reads the commits before it can build the next step
 
     for _ in range(warmup):
         one()
     torch.cuda.synchronize()
     if sampler:
-        sampler.tag = "e2e"
+        sampler.tag = "e2e_" + mode
     t0 = time.perf_counter()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     start.record()
@@ -390,6 +432,16 @@ def reduce_over_ranks(times_ms, counts, device):
     return [float(x) for x in t.tolist()], [float(x) for x in c.tolist()]
 
 
+def tensor_peaks():
+    """Measured bf16 GEMM throughput on this machine (burst and sustained), or the stated fallback."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            p = json.load(f)
+        return float(p["bf16_tflops"]), float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "measured"
+    except Exception:
+        return 1590.0, 1400.0, "fallback"
+
+
 def run_product(args):
     import torch
     import torch.distributed as dist
@@ -412,7 +464,7 @@ def run_product(args):
     w.load_library()
 
     sampler = ClockSampler(local) if rank == 0 else None
-    n_state = args.steps + args.warmup
+    n_state = max(args.steps, args.warmup)
     wl = Workload(args.workload, rank_seed(rank), args.attn, n_state, args.batch, args.temperature)
     if sampler:
         sampler.start()
@@ -423,39 +475,85 @@ def run_product(args):
         torch.cuda.synchronize()
 
     barrier()
-    ms, attn_ms, committed, launches = time_workload(wl, args.steps, args.warmup, sampler)
+    t = time_workload(wl, args.steps, args.warmup, sampler, min_region_s=args.min_seconds)
     barrier()
-    (ms, attn_ms), (committed_total,) = reduce_over_ranks([ms, attn_ms], [committed], "cuda")
+    (ms, ms_median, ms_best, attn_ms), (committed_total,) = reduce_over_ranks(
+        [t["ms"], t["ms_median"], t["ms_best"], t["attn_ms"]], [t["committed"]], "cuda")
+    launches = t["launches"]
     assert int(wl.step.status.item()) == 0, "device status word set during the benchmark"
 
-    if args.no_e2e:
-        e2e_ms, e2e_committed, h2d, d2h = float("nan"), 0, 0, 0
-    else:
-        e2e_ms, e2e_committed, h2d, d2h = time_e2e(wl, max(3, min(args.steps, 10)), 3, sampler)
-    (e2e_ms,), (e2e_committed,) = reduce_over_ranks([e2e_ms], [e2e_committed], "cuda")
+    # end to end from host buffers: hidden states in (LM head inside the step), and the logits-from-host variant
+    e2e = {"lmhead": None, "logits": None}
+    if not args.no_e2e and wl.cfg.dtype == "bf16":
+        hidden = 4096
+        g = torch.Generator(device="cuda").manual_seed(rank_seed(rank))
+        lm_head = (torch.randn(wl.cfg.vocab, hidden, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+        e2e["lmhead"] = time_e2e(wl, max(3, min(args.steps, 10)), 3, sampler, "lmhead", hidden, lm_head)
+        del lm_head
+        torch.cuda.empty_cache()
+        e2e["logits"] = time_e2e(wl, max(3, min(args.steps, 10)), 3, sampler, "logits")
+    elif not args.no_e2e:
+        e2e["logits"] = time_e2e(wl, max(3, min(args.steps, 10)), 3, sampler, "logits")
+    e2e_json = {}
+    for mode, r in e2e.items():
+        r = r or (float("nan"), 0, 0, 0)
+        (e_ms,), (e_commit,) = reduce_over_ranks([r[0]], [r[1]], "cuda")
+        e2e_json[mode] = {"value": (e_commit / (e_ms * 1e-3)) if e_ms == e_ms else None, "unit": UNIT, "ms_per_step": e_ms,
+                          "h2d_bytes_per_step": r[2], "d2h_bytes_per_step": r[3]}
+    e2e_json["lmhead"]["call"] = "wedlm_step_host_lmhead: hidden states [B,W,4096] from pinned host memory, output embedding resident"
+    e2e_json["logits"]["call"] = "wedlm_step_host: logits rows of the mask slots from pinned host memory"
 
     graph_ms = time_graph(wl, args.steps, args.warmup) if world == 1 else None
-    others = {}
-    cpu = None
+    peak, peak_kind = measured_peaks()
+    tf_burst, tf_sustained, tf_kind = tensor_peaks()
+    others, extras, cpu = {}, {}, None
     if rank == 0 and world == 1 and not args.no_extras:
         for name in ("cfg2_qwen_b1", "cfg4_long"):
             if name == args.workload:
                 continue
             try:
                 o = Workload(name, BASE_SEED, args.attn, n_state)
-                oms, oattn, ocommit, _ = time_workload(o, args.steps, args.warmup, sampler, tag="other")
+                ot = time_workload(o, args.steps, args.warmup, sampler, tag=name, min_region_s=0.4 * args.min_seconds)
                 ob = o.bytes
                 gms = time_graph(o, args.steps, args.warmup)
+                a_ms = ot["attn_ms"]
                 others[name] = {
-                    "ms_per_step": oms, "committed_tokens_per_s": ocommit / (oms * 1e-3),
+                    "ms_per_step": ot["ms"], "ms_per_step_median": ot["ms_median"], "ms_per_step_best": ot["ms_best"],
+                    "timed_region_s": ot["region_s"], "timed_blocks": ot["blocks"],
+                    "committed_tokens_per_s": ot["committed"] / (ot["ms"] * 1e-3),
                     "cuda_graph_ms_per_step": gms, "cuda_graph_l2": "cold" if o.n_copies == 1 else "warm",
-                    "attn_kernel_ms": oattn, "attn_kernel_GBps": ob["attn_kernel"] / (oattn * 1e-3) / 1e9,
-                    "rotating_copies": o.n_copies,
+                    "attn_kernel_ms": a_ms, "attn_kernel_GBps": ob["attn_kernel"] / (a_ms * 1e-3) / 1e9,
+                    "rotating_copies": o.n_copies, "clocks": sampler.summary(name) if sampler else None,
+                    # the attention kernel against both roofs (this shape sits on the ridge)
+                    "roofline": {
+                        "kernel": "window attention", "kernel_ms": a_ms,
+                        "hbm": {"algorithmic_bytes": ob["attn_kernel"], "achieved_GBps": ob["attn_kernel"] / (a_ms * 1e-3) / 1e9,
+                                "peak_GBps": peak, "frac": ob["attn_kernel"] / (a_ms * 1e-3) / 1e9 / peak,
+                                "frac_of_nominal_8TBps": ob["attn_kernel"] / (a_ms * 1e-3) / 1e9 / 8000.0},
+                        "tensor": {"flops": ob["attn_flops"], "achieved_TFLOPs": ob["attn_flops"] / (a_ms * 1e-3) / 1e12,
+                                   "peak_TFLOPs_burst": tf_burst, "peak_TFLOPs_sustained": tf_sustained,
+                                   "frac_of_burst": ob["attn_flops"] / (a_ms * 1e-3) / 1e12 / tf_burst,
+                                   "frac_of_sustained": ob["attn_flops"] / (a_ms * 1e-3) / 1e12 / tf_sustained,
+                                   "peak_kind": tf_kind}},
                 }
                 del o
                 torch.cuda.empty_cache()
             except Exception as e:      # pragma: no cover
                 others[name] = {"error": repr(e)}
+        # short legs of the other parts of the library, so that every measured claim has a line here
+        for key, fn in (("lmhead", lambda: measure_lmhead(args.steps, args.warmup)),
+                        ("dual_stream", lambda: measure_dual_stream(["ds_4k"], args.attn, args.steps, args.warmup)),
+                        ("cfg5_loop", lambda: measure_loop_short(args))):
+            try:
+                if sampler:
+                    sampler.tag = key
+                extras[key] = fn()
+                if sampler:
+                    extras[key]["clocks"] = sampler.summary(key)
+                    sampler.tag = "other"
+                torch.cuda.empty_cache()
+            except Exception as e:      # pragma: no cover
+                extras[key] = {"error": repr(e)}
     if sampler:
         sampler.stop()
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -471,10 +569,11 @@ def run_product(args):
                          f"({dt:.1f}s of CPU wall time)"}
 
     if rank == 0:
-        peak, peak_kind = measured_peaks()
         bts = wl.bytes
         achieved = bts["attn_kernel"] / (attn_ms * 1e-3) / 1e9
         key = f"{wl.cfg.name}:{args.attn}"
+        clocks = sampler.summary("timed") if sampler else None
+        head_e2e = e2e_json["lmhead"] if e2e_json["lmhead"]["value"] is not None else e2e_json["logits"]
         line = {
             "metric": METRIC, "value": committed_total / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
@@ -486,9 +585,14 @@ def run_product(args):
                        "committed_tokens_per_step": committed_total,
                        "sample": "argmax" if args.temperature <= 0 else f"gumbel_max_T{args.temperature:g}",
                        "kv_stream_bytes": bts["kv_stream"], "logits_stream_bytes": bts["logits_stream"]},
-            "clocks": sampler.summary() if sampler else None,
-            "e2e": {"value": e2e_committed / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            # steady state: blocks of `steps` steps repeated back to back until the timed region is long enough for the
+            # clocks to settle; ms_per_step (and value) is the mean over the whole region
+            "timing": {"timed_blocks": t["blocks"], "timed_region_s": t["region_s"], "steps_per_block": args.steps,
+                       "ms_per_step_median": ms_median, "ms_per_step_best": ms_best,
+                       "ms_x_sm_mhz": (ms * clocks["sm_mhz"]) if clocks and clocks.get("sm_mhz") else None},
+            "clocks": clocks,
+            "e2e": head_e2e,
+            "e2e_logits_host": e2e_json["logits"],
             "gpu_launches": int(launches),
             "cuda_graph": None if graph_ms is None else {"ms_per_step": graph_ms, "value": committed_total / (graph_ms * 1e-3),
                                                          "note": "same step replayed from one captured graph"},
@@ -498,7 +602,10 @@ def run_product(args):
                          "traffic": (NCU_TRAFFIC_RATIO[key] * bts["attn_kernel"] if key in NCU_TRAFFIC_RATIO and not args.batch else None),
                          "traffic_note": "ncu dram bytes of a batch-16 capture scaled by algorithmic bytes",
                          "kernel_ms": attn_ms,
-                         "algorithmic_bytes": bts["attn_kernel"]},
+                         "algorithmic_bytes": bts["attn_kernel"],
+                         "bytes_definition": "K and V of every cached prefix token AND of the staged window rows (4096 B per token), "
+                                             "plus the rotated q read and the output write",
+                         "frac_prefix_tokens_only": bts["kv_prefix_only"] / (attn_ms * 1e-3) / 1e9 / peak},
             "step_hbm": {"note": "whole step: K/V and logits streams plus q/out, against the same measured peak",
                          "algorithmic_bytes": bts["attn_kernel"] + bts["logits_stream"],
                          "achieved": (bts["attn_kernel"] + bts["logits_stream"]) / (ms * 1e-3) / 1e9, "unit": "GB/s",
@@ -506,6 +613,7 @@ def run_product(args):
             "cpu_baseline": cpu,
             "other_workloads": others,
         }
+        line.update(extras)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
@@ -516,7 +624,29 @@ def run_product(args):
 # ----------------------------------------------------------------------------------------------
 # end-to-end streaming decode loop (the 4-layer configuration); not the default bench line
 # ----------------------------------------------------------------------------------------------
+def measure_loop_short(args):
+    """The end-to-end loop in a form short enough for the default line: 256 new tokens per sequence at the
+    calibrated tilt lse + 8, streaming commits, W = 16 against the same harness at W = 2 and W = 1."""
+    import types
+    a = types.SimpleNamespace(**vars(args))
+    a.loop_new_tokens, a.loop_windows, a.loop_block_windows, a.loop_fused_windows = 256, [16, 2, 1], [], []
+    a.loop_tilts, a.loop_eager = [("lse", 8.0)], False
+    line = measure_loop(a)
+    by_w = {r["window"]: r for r in line["results"]}
+    out = {"config": line["config"], "results": line["results"], "unit": "generated tokens/s"}
+    if 16 in by_w and 1 in by_w:
+        out["speedup_w16_over_w1"] = by_w[16]["tokens_per_s"] / by_w[1]["tokens_per_s"]
+    if 16 in by_w and 2 in by_w:
+        out["speedup_w16_over_w2"] = by_w[16]["tokens_per_s"] / by_w[2]["tokens_per_s"]
+    return out
+
+
 def run_loop(args):
+    print(json.dumps(measure_loop(args)), flush=True)
+    return 0
+
+
+def measure_loop(args):
     """Random-init 4-layer model of Qwen3-8B width, batch 16, 512-token prompt, 1024 new tokens per
     sequence, LM-head logits tilted toward a seeded target sequence.  Generated tokens/s, steps and
     p_cache (Eq. 4) for W = 16 against the same harness at W = 1 and W = 2, for every tilt."""
@@ -586,11 +716,16 @@ def run_loop(args):
                        "hidden": H, "lse_of_untilted_logits": lse0,
                        "timing": "host wall clock around generate(), includes the graph capture and the per-step read-back of commits"},
             "results": results}
-    print(json.dumps(line), flush=True)
-    return 0
+    del wts, lm_head_vh
+    return line
 
 
 def run_lmhead(args):
+    print(json.dumps(measure_lmhead(args.steps, args.warmup)), flush=True)
+    return 0
+
+
+def measure_lmhead(steps, warmup):
     """LM head + confidence/commit at the end-to-end configuration's shape (16 x 16 rows, hidden 4096, vocabulary
     151 936): the fused call (logits stay in tensor memory) against a library GEMM that writes bf16 logits
     followed by the streaming confidence call."""
@@ -624,7 +759,7 @@ def run_lmhead(args):
     out = {}
     for name, fn in (("fused", fused), ("gemm_then_confidence", unfused)):
         ts = []
-        for _ in range(args.warmup + args.steps):
+        for _ in range(warmup + steps):
             f, t, p = filled.clone(), tok.clone(), pl.clone()
             a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
@@ -632,22 +767,26 @@ def run_lmhead(args):
             e.record()
             torch.cuda.synchronize()
             ts.append(a.elapsed_time(e))
-        ts = ts[args.warmup:]
+        ts = ts[warmup:]
         out[name] = {"ms_min": min(ts), "ms_median": statistics.median(ts)}
     weights = V * H * 2
     line = {"metric": "lm_head_confidence_ms", "unit": "ms", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": "lmhead", "rows": B * W, "hidden": H, "vocab": V},
             "results": out, "weight_bytes": weights, "flops": 2 * B * W * H * V,
-            "fused_weight_stream_GBps": weights / (out["fused"]["ms_median"] * 1e-3) / 1e9}
-    print(json.dumps(line), flush=True)
-    return 0
+            "fused_weight_stream_GBps": weights / (out["fused"]["ms_median"] * 1e-3) / 1e9,
+            "fused_TFLOPs": 2 * B * W * H * V / (out["fused"]["ms_median"] * 1e-3) / 1e12}
+    return line
 
 
 # ----------------------------------------------------------------------------------------------
 # Dual-Stream Masking training forward (Section 4.2): attention over the two-stream input
 # ----------------------------------------------------------------------------------------------
 def run_dual_stream(args):
-    import statistics
+    print(json.dumps(measure_dual_stream(args.ds_configs, args.attn, args.steps, args.warmup)), flush=True)
+    return 0
+
+
+def measure_dual_stream(ds_configs, attn, steps, warmup):
     import torch
     from paper_2512_22737_b200 import build as b
     from workloads import DS_CONFIGS, make_dual_stream
@@ -655,12 +794,12 @@ def run_dual_stream(args):
     import paper_2512_22737_b200 as w
     torch.cuda.set_device(0)
     out = {}
-    for name in args.ds_configs:
+    for name in ds_configs:
         c = DS_CONFIGS[name]
         inp = make_dual_stream(c)
         cfg = w.make_config(batch=c.n_seq, window=c.block, n_q_heads=c.n_q_heads, n_kv_heads=c.n_kv_heads,
                             head_dim=c.head_dim, page_size=c.page_size, vocab=c.vocab, dtype=c.dtype,
-                            rope_theta=c.rope_theta, mask_token_id=c.mask_token_id, attn_impl=args.attn)
+                            rope_theta=c.rope_theta, mask_token_id=c.mask_token_id, attn_impl=attn)
         N, K, L, B, Lp = c.n_seq, c.n_blocks, c.seq_len, c.block, c.padded_len
         i32 = dict(dtype=torch.int32, device="cuda")
         tokens, masked = w.to_device(inp["tokens"]), w.to_device(inp["masked"])
@@ -671,7 +810,7 @@ def run_dual_stream(args):
         status = torch.zeros(1, **i32)
         flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")       # larger than L2
         ts, launches0 = [], w.wedlm_launch_count()
-        for it in range(args.warmup + args.steps):
+        for it in range(warmup + steps):
             flush.fill_(it & 0xff)
             a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
@@ -681,8 +820,8 @@ def run_dual_stream(args):
             torch.cuda.synchronize()
             ts.append(a.elapsed_time(e))
         assert int(status.item()) == 0
-        launches = (w.wedlm_launch_count() - launches0) // (args.warmup + args.steps)
-        ts = ts[args.warmup:]
+        launches = (w.wedlm_launch_count() - launches0) // (warmup + steps)
+        ts = ts[warmup:]
         ms = statistics.median(ts)
         # visible keys per row: k*B + r + 1, both streams; QK^T and PV are 2*D flops per (row, key, head) each
         keys = 2 * sum((i // B) * B + (i % B) + 1 for i in range(L))
@@ -697,15 +836,14 @@ def run_dual_stream(args):
             peak, kind = float(json.load(f)["bf16_tflops"]), "measured"
     except Exception:
         peak, kind = 1590.0, "fallback"
-    first = out[args.ds_configs[0]]
+    first = out[ds_configs[0]]
     line = {"metric": "dual_stream_attention_tokens_per_s", "value": first["tokens_per_s"], "unit": "tokens/s", "n_gpus": 1,
             "dtype": "bf16", "data": "synthetic", "higher_is_better": True,
-            "config": {"workload": args.ds_configs[0], "l2": "flushed between iterations", "attn_impl": args.attn},
+            "config": {"workload": ds_configs[0], "l2": "flushed between iterations", "attn_impl": attn},
             "roofline": {"bound": "tensor", "achieved": first["attention_TFLOPs"], "peak": peak, "peak_kind": kind,
                          "unit": "TFLOP/s", "frac": first["attention_TFLOPs"] / peak, "traffic": None},
             "results": out}
-    print(json.dumps(line), flush=True)
-    return 0
+    return line
 
 
 def main():
@@ -720,6 +858,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing (profiling runs)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling runs)")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="blocks of --steps steps are repeated until the timed region is at least this long")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="Sample() temperature of the step workloads (0 = arg-max, the headline configuration)")
     ap.add_argument("--ds-configs", type=lambda s: s.split(","), default=["ds_4k", "ds_8k"],

@@ -15,7 +15,8 @@
  *                            selection by distance-adjusted entropy (Eq. 11), then Commit,
  *                            Predict and Refill of Algorithm 1.
  *   wedlm_window_refill      Commit + shift + Refill alone.
- *   wedlm_step_host          the three calls above for step inputs that live in host memory.
+ *   wedlm_step_host          the three calls above for step inputs that live in host memory
+ *   wedlm_step_host_lmhead   (logits from the host, or hidden states from the host with the LM head on the device).
  *   wedlm_dual_stream_*      training side (Section 4.2): two-stream input construction and its attention.
  *
  * Conventions common to every call
@@ -340,6 +341,27 @@ int wedlm_step_host(const wedlm_config_t* cfg, uint8_t* h_filled, int32_t* h_win
                     void* k_cache, void* v_cache, int32_t* h_committed_tokens, int32_t* h_committed_count,
                     int32_t* h_filled_count, void* workspace, size_t workspace_bytes, void** attn_out,
                     int32_t* status, void* stream);
+
+/*
+ * The same step with the LM head inside it (Algorithm 1, "(l, K_W, V_W) <- Forward(W, K, V)" followed by Predict):
+ * instead of [B,W,V] logits the host hands over the hidden states of the window rows, and the output embedding
+ * stays resident on the device.  The confidence pass is wedlm_lmhead_confidence_commit, so no logits ever exist
+ * and the per-step traffic over the host link shrinks from B*W*V to B*W*hidden elements.  bf16 only.
+ *   hidden            H (multiple of 64)
+ *   h_hidden_states   host, in  bf16 [B,W,H] physical order (all rows are sent)
+ *   lm_head           device, in bf16 [V,H]
+ *   h_tilt_ids, tilt  host i32 [B,W] or NULL, and the additive tilt (as in wedlm_lmhead_confidence_commit)
+ * Everything else as in wedlm_step_host; workspace of wedlm_step_host_lmhead_workspace_bytes(cfg, hidden) bytes.
+ * cfg->sample_temperature must be 0.
+ */
+size_t wedlm_step_host_lmhead_workspace_bytes(const wedlm_config_t* cfg, int32_t hidden);
+int wedlm_step_host_lmhead(const wedlm_config_t* cfg, int32_t hidden, uint8_t* h_filled, int32_t* h_window_tokens,
+                           int32_t* h_prefix_len, int32_t* h_window_len, int32_t* h_remaining_budget,
+                           const int32_t* h_block_table, const void* h_q, const void* h_k, const void* h_v,
+                           const void* h_hidden_states, const void* lm_head, const int32_t* h_tilt_ids, float tilt,
+                           void* k_cache, void* v_cache, int32_t* h_committed_tokens, int32_t* h_committed_count,
+                           int32_t* h_filled_count, void* workspace, size_t workspace_bytes, void** attn_out,
+                           int32_t* status, void* stream);
 
 /*
  * Dual-Stream Masking for training (Section 4.2): the forward-pass pieces that need no data or weights.

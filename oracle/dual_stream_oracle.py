@@ -96,3 +96,31 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, p_input: np.ndarray, 
             p /= p.sum()
             out[a, h] = p @ vf[cols, g]
     return out
+
+
+def attention_dense(q: np.ndarray, k: np.ndarray, v: np.ndarray, p_input: np.ndarray, block: int, *, theta: float,
+                    rope_style: int = 0, scale: Optional[float] = None) -> np.ndarray:
+    """The same quantity as `attention`, for all 2L rows at once: per head one dense score matrix over all
+    2L x 2L (row, key) pairs, the pairs outside `visibility(L, block)` set to -inf, a row-wise softmax and one
+    product with V.  It is the definition with the mask written as a matrix instead of as a list of columns
+    per row; used where every row of a long sequence is compared (the row-by-row form takes minutes there)."""
+    qf, kf, vf = to_f64(q), to_f64(k), to_f64(v)
+    N, Hq, D = qf.shape
+    L = N // 2
+    G = Hq // kf.shape[1]
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    pos = np.asarray(p_input)
+    q_rot = rope(qf, pos[:, None], theta, rope_style)
+    k_rot = rope(kf, pos[:, None], theta, rope_style)
+    vis = visibility(L, block)
+    out = np.zeros((N, Hq, D))
+    for h in range(Hq):
+        g = h // G
+        s = scale * (q_rot[:, h] @ k_rot[:, g].T)
+        s[~vis] = -np.inf
+        s -= s.max(axis=1, keepdims=True)
+        np.exp(s, out=s)
+        s /= s.sum(axis=1, keepdims=True)
+        out[:, h] = s @ vf[:, g]
+    return out

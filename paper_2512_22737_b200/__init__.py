@@ -28,6 +28,8 @@ from .binding import (  # noqa: F401
     wedlm_reorder,
     wedlm_selftest_wait_expiry,
     wedlm_step_host,
+    wedlm_step_host_lmhead,
+    wedlm_step_host_lmhead_workspace_bytes,
     wedlm_step_host_workspace_bytes,
     wedlm_strerror,
     wedlm_version,

@@ -105,6 +105,11 @@ def load_library() -> ctypes.CDLL:
     lib.wedlm_step_host_workspace_bytes.argtypes = [cfgp]
     lib.wedlm_step_host.restype = ctypes.c_int
     lib.wedlm_step_host.argtypes = [cfgp] + [vp] * 15 + [vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_void_p), i32p, vp]
+    lib.wedlm_step_host_lmhead_workspace_bytes.restype = ctypes.c_size_t
+    lib.wedlm_step_host_lmhead_workspace_bytes.argtypes = [cfgp, ctypes.c_int32]
+    lib.wedlm_step_host_lmhead.restype = ctypes.c_int
+    lib.wedlm_step_host_lmhead.argtypes = [cfgp, ctypes.c_int32] + [vp] * 12 + [ctypes.c_float] + [vp] * 5 + \
+                                          [vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_void_p), i32p, vp]
     lib.wedlm_dual_stream_construct.restype = ctypes.c_int
     lib.wedlm_dual_stream_construct.argtypes = [cfgp, ctypes.c_int32, ctypes.c_int32, i32p, u8p, i32p, i32p, u8p, i32p, vp]
     lib.wedlm_dual_stream_workspace_bytes.restype = ctypes.c_size_t
@@ -335,6 +340,31 @@ def wedlm_step_host(cfg, h_filled, h_window_tokens, h_prefix_len, h_window_len, 
         _hptr(h_filled_count, i32, "h_filled_count"), _ptr(workspace, None, "workspace"),
         ctypes.c_size_t(workspace.numel() * workspace.element_size()), ctypes.byref(out_ptr),
         _ptr(status, i32, "status"), _stream(stream)), "wedlm_step_host")
+    return int(out_ptr.value or 0)
+
+
+def wedlm_step_host_lmhead_workspace_bytes(cfg, hidden: int) -> int:
+    return int(load_library().wedlm_step_host_lmhead_workspace_bytes(ctypes.byref(cfg), ctypes.c_int32(hidden)))
+
+
+def wedlm_step_host_lmhead(cfg, h_filled, h_window_tokens, h_prefix_len, h_window_len, h_remaining_budget, h_block_table,
+                           h_q, h_k, h_v, h_hidden_states, lm_head, h_tilt_ids, tilt, k_cache, v_cache, h_committed_tokens,
+                           h_committed_count, h_filled_count, workspace, status=None, stream=None) -> int:
+    """One whole step from host tensors with the LM head inside it: hidden states [B,W,H] come from the host, the
+    output embedding [V,H] is a device tensor.  Returns the device address of the attention output."""
+    i32, u8 = torch.int32, torch.uint8
+    out_ptr = ctypes.c_void_p()
+    _check(load_library().wedlm_step_host_lmhead(
+        ctypes.byref(cfg), ctypes.c_int32(h_hidden_states.shape[-1]), _hptr(h_filled, u8, "h_filled"),
+        _hptr(h_window_tokens, i32, "h_window_tokens"), _hptr(h_prefix_len, i32, "h_prefix_len"),
+        _hptr(h_window_len, i32, "h_window_len"), _hptr(h_remaining_budget, i32, "h_remaining_budget"),
+        _hptr(h_block_table, i32, "h_block_table"), _hptr(h_q, None, "h_q"), _hptr(h_k, None, "h_k"), _hptr(h_v, None, "h_v"),
+        _hptr(h_hidden_states, None, "h_hidden_states"), _ptr(lm_head, torch.bfloat16, "lm_head"),
+        _hptr(h_tilt_ids, i32, "h_tilt_ids"), ctypes.c_float(tilt), _ptr(k_cache, cfg.torch_dtype, "k_cache"),
+        _ptr(v_cache, cfg.torch_dtype, "v_cache"), _hptr(h_committed_tokens, i32, "h_committed_tokens"),
+        _hptr(h_committed_count, i32, "h_committed_count"), _hptr(h_filled_count, i32, "h_filled_count"),
+        _ptr(workspace, None, "workspace"), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+        ctypes.byref(out_ptr), _ptr(status, i32, "status"), _stream(stream)), "wedlm_step_host_lmhead")
     return int(out_ptr.value or 0)
 
 

@@ -385,13 +385,15 @@ int wedlm_dual_stream_attn(const wedlm_config_t* cfg, int32_t n_blocks, const vo
 namespace {
 
 struct HostStepPlan {
-  size_t off_filled, off_tokens, off_prefix, off_wlen, off_budget, off_table, off_q, off_k, off_v, off_logits;
+  size_t off_filled, off_tokens, off_prefix, off_wlen, off_budget, off_table, off_q, off_k, off_v, off_logits, off_tilt;
   size_t off_perm, off_inv, off_pos, off_tokphys, off_nfilled, off_ncommit, off_out, off_argmax, off_maxprob, off_entropy,
       off_lse, off_ctok, off_ccount, off_fcount, off_attn_ws, off_conf_ws;
   size_t attn_ws_bytes, conf_ws_bytes, total;
 };
 
-int plan_host_step(const wedlm_config_t* cfg, HostStepPlan* out) {
+// hidden == 0: the step takes logits [B,W,V]; hidden > 0: it takes hidden states [B,W,hidden] (and per-row tilt ids)
+// and the confidence pass is the fused LM-head call
+int plan_host_step(const wedlm_config_t* cfg, int32_t hidden, HostStepPlan* out) {
   int rc = check_config(cfg, true, true);
   if (rc != WEDLM_OK) return rc;
   const size_t B = cfg->batch, W = cfg->window, elem = cfg->dtype == WEDLM_DTYPE_BF16 ? 2 : 4;
@@ -407,7 +409,8 @@ int plan_host_step(const wedlm_config_t* cfg, HostStepPlan* out) {
   p.off_q = take(B * W * cfg->n_q_heads * cfg->head_dim * elem);
   p.off_k = take(B * W * cfg->n_kv_heads * cfg->head_dim * elem);
   p.off_v = take(B * W * cfg->n_kv_heads * cfg->head_dim * elem);
-  p.off_logits = take(B * W * (size_t)cfg->vocab * elem);
+  p.off_logits = hidden > 0 ? take(B * W * (size_t)hidden * elem) : take(B * W * (size_t)cfg->vocab * elem);
+  p.off_tilt = take(B * W * 4);
   p.off_perm = take(B * W * 4);
   p.off_inv = take(B * W * 4);
   p.off_pos = take(B * W * 4);
@@ -423,7 +426,7 @@ int plan_host_step(const wedlm_config_t* cfg, HostStepPlan* out) {
   p.off_ccount = take(B * 4);
   p.off_fcount = take(B * 4);
   p.attn_ws_bytes = plan_attention(cfg).total_bytes;
-  p.conf_ws_bytes = confidence_workspace_bytes(cfg);
+  p.conf_ws_bytes = hidden > 0 ? wedlm_lmhead_confidence_workspace_bytes(cfg) : confidence_workspace_bytes(cfg);
   p.off_attn_ws = take(p.attn_ws_bytes);
   p.off_conf_ws = take(p.conf_ws_bytes);
   p.total = at;
@@ -435,23 +438,36 @@ int plan_host_step(const wedlm_config_t* cfg, HostStepPlan* out) {
 
 size_t wedlm_step_host_workspace_bytes(const wedlm_config_t* cfg) {
   HostStepPlan p;
-  if (plan_host_step(cfg, &p) != WEDLM_OK) return 0;
+  if (plan_host_step(cfg, 0, &p) != WEDLM_OK) return 0;
   return p.total;
 }
 
-int wedlm_step_host(const wedlm_config_t* cfg, uint8_t* h_filled, int32_t* h_window_tokens, int32_t* h_prefix_len,
-                    int32_t* h_window_len, int32_t* h_remaining_budget, const int32_t* h_block_table, const void* h_q,
-                    const void* h_k, const void* h_v, const void* h_logits, void* k_cache, void* v_cache,
-                    int32_t* h_committed_tokens, int32_t* h_committed_count, int32_t* h_filled_count, void* workspace,
-                    size_t workspace_bytes, void** attn_out, int32_t* status, void* stream) {
+size_t wedlm_step_host_lmhead_workspace_bytes(const wedlm_config_t* cfg, int32_t hidden) {
   HostStepPlan p;
-  int rc = plan_host_step(cfg, &p);
+  if (hidden < 64 || hidden % 64 != 0 || plan_host_step(cfg, hidden, &p) != WEDLM_OK) return 0;
+  return p.total;
+}
+
+namespace {
+
+// Both host-step calls: logits from the host (h_hidden == NULL) or hidden states from the host with the output
+// embedding resident on the device.
+int step_host_impl(const wedlm_config_t* cfg, int32_t hidden, uint8_t* h_filled, int32_t* h_window_tokens,
+                   int32_t* h_prefix_len, int32_t* h_window_len, int32_t* h_remaining_budget, const int32_t* h_block_table,
+                   const void* h_q, const void* h_k, const void* h_v, const void* h_logits, const void* h_hidden,
+                   const void* lm_head, const int32_t* h_tilt_ids, float tilt, void* k_cache, void* v_cache,
+                   int32_t* h_committed_tokens, int32_t* h_committed_count, int32_t* h_filled_count, void* workspace,
+                   size_t workspace_bytes, void** attn_out, int32_t* status, void* stream) {
+  HostStepPlan p;
+  int rc = plan_host_step(cfg, hidden, &p);
   if (rc != WEDLM_OK) return rc;
   if (attn_out) *attn_out = nullptr;
   if (cfg->batch == 0) return WEDLM_OK;
-  if (!h_filled || !h_window_tokens || !h_prefix_len || !h_block_table || !h_q || !h_k || !h_v || !h_logits || !k_cache ||
+  const bool fused = hidden > 0;
+  if (!h_filled || !h_window_tokens || !h_prefix_len || !h_block_table || !h_q || !h_k || !h_v || !k_cache ||
       !v_cache || !h_committed_tokens || !h_committed_count || !workspace)
     return WEDLM_ERR_INVALID_ARG;
+  if (fused ? (!h_hidden || !lm_head) : !h_logits) return WEDLM_ERR_INVALID_ARG;
   if (!aligned16(workspace) || !aligned16(k_cache) || !aligned16(v_cache)) return WEDLM_ERR_INVALID_ARG;
   if (workspace_bytes < p.total) return WEDLM_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
@@ -480,7 +496,7 @@ int wedlm_step_host(const wedlm_config_t* cfg, uint8_t* h_filled, int32_t* h_win
   int32_t* d_pos = reinterpret_cast<int32_t*>(ws + p.off_pos);
   int32_t* d_nfilled = reinterpret_cast<int32_t*>(ws + p.off_nfilled);
   int32_t* d_ncommit = reinterpret_cast<int32_t*>(ws + p.off_ncommit);
-  // reorder and attention need only the small inputs; the logits follow
+  // reorder and attention need only the small inputs; the logits / hidden states follow
   rc = wedlm_reorder(cfg, d_filled, d_tokens, d_prefix, d_wlen, d_perm, reinterpret_cast<int32_t*>(ws + p.off_inv), d_pos,
                      reinterpret_cast<int32_t*>(ws + p.off_tokphys), d_nfilled, d_ncommit, stream);
   if (rc != WEDLM_OK) return rc;
@@ -488,25 +504,40 @@ int wedlm_step_host(const wedlm_config_t* cfg, uint8_t* h_filled, int32_t* h_win
                          reinterpret_cast<int32_t*>(ws + p.off_table), d_prefix, d_pos, ws + p.off_out, nullptr,
                          ws + p.off_attn_ws, p.attn_ws_bytes, status, stream);
   if (rc != WEDLM_OK) return rc;
-  // Logits: only the rows the confidence pass reads.  After reordering the mask rows of a sequence are the
-  // physical rows [n_filled, window_len), one contiguous range, and n_filled is a count over the host's flags.
-  for (size_t b = 0; b < B; ++b) {
-    long long L = h_window_len ? h_window_len[b] : (long long)W;
-    L = L < 0 ? 0 : (L > (long long)W ? (long long)W : L);
-    long long nf = 0;
-    for (long long j = 0; j < L; ++j) nf += h_filled[b * W + j] != 0;
-    if (L > nf) {
-      const size_t off = (b * W + (size_t)nf) * (size_t)cfg->vocab * elem;
-      if (!up(p.off_logits + off, static_cast<const char*>(h_logits) + off, (size_t)(L - nf) * cfg->vocab * elem))
-        return WEDLM_ERR_CUDA;
+  int32_t* d_argmax = reinterpret_cast<int32_t*>(ws + p.off_argmax);
+  float* d_maxprob = reinterpret_cast<float*>(ws + p.off_maxprob);
+  float* d_entropy = reinterpret_cast<float*>(ws + p.off_entropy);
+  float* d_lse = reinterpret_cast<float*>(ws + p.off_lse);
+  int32_t* d_ctok = reinterpret_cast<int32_t*>(ws + p.off_ctok);
+  int32_t* d_ccount = reinterpret_cast<int32_t*>(ws + p.off_ccount);
+  int32_t* d_fcount = reinterpret_cast<int32_t*>(ws + p.off_fcount);
+  if (fused) {
+    // hidden states of all rows (the tensor-core tiles span whole row blocks), tilt ids if any
+    if (!up(p.off_logits, h_hidden, B * W * (size_t)hidden * elem)) return WEDLM_ERR_CUDA;
+    if (h_tilt_ids && !up(p.off_tilt, h_tilt_ids, B * W * 4)) return WEDLM_ERR_CUDA;
+    rc = wedlm_lmhead_confidence_commit(cfg, hidden, ws + p.off_logits, lm_head,
+                                        h_tilt_ids ? reinterpret_cast<int32_t*>(ws + p.off_tilt) : nullptr, tilt, d_perm,
+                                        d_nfilled, d_ncommit, d_tokens, d_filled, d_prefix, d_wlen, d_budget, d_argmax,
+                                        d_maxprob, d_entropy, d_lse, d_ctok, d_ccount, d_fcount, ws + p.off_conf_ws,
+                                        p.conf_ws_bytes, status, stream);
+  } else {
+    // Logits: only the rows the confidence pass reads.  After reordering the mask rows of a sequence are the
+    // physical rows [n_filled, window_len), one contiguous range, and n_filled is a count over the host's flags.
+    for (size_t b = 0; b < B; ++b) {
+      long long L = h_window_len ? h_window_len[b] : (long long)W;
+      L = L < 0 ? 0 : (L > (long long)W ? (long long)W : L);
+      long long nf = 0;
+      for (long long j = 0; j < L; ++j) nf += h_filled[b * W + j] != 0;
+      if (L > nf) {
+        const size_t off = (b * W + (size_t)nf) * (size_t)cfg->vocab * elem;
+        if (!up(p.off_logits + off, static_cast<const char*>(h_logits) + off, (size_t)(L - nf) * cfg->vocab * elem))
+          return WEDLM_ERR_CUDA;
+      }
     }
+    rc = wedlm_confidence_commit(cfg, ws + p.off_logits, d_perm, d_nfilled, d_ncommit, d_tokens, d_filled, d_prefix, d_wlen,
+                                 d_budget, d_argmax, d_maxprob, d_entropy, d_lse, d_ctok, d_ccount, d_fcount,
+                                 ws + p.off_conf_ws, p.conf_ws_bytes, status, stream);
   }
-  rc = wedlm_confidence_commit(cfg, ws + p.off_logits, d_perm, d_nfilled, d_ncommit, d_tokens, d_filled, d_prefix, d_wlen,
-                               d_budget, reinterpret_cast<int32_t*>(ws + p.off_argmax),
-                               reinterpret_cast<float*>(ws + p.off_maxprob), reinterpret_cast<float*>(ws + p.off_entropy),
-                               reinterpret_cast<float*>(ws + p.off_lse), reinterpret_cast<int32_t*>(ws + p.off_ctok),
-                               reinterpret_cast<int32_t*>(ws + p.off_ccount), reinterpret_cast<int32_t*>(ws + p.off_fcount),
-                               ws + p.off_conf_ws, p.conf_ws_bytes, status, stream);
   if (rc != WEDLM_OK) return rc;
   ok = down(h_committed_tokens, p.off_ctok, B * W * 4) && down(h_committed_count, p.off_ccount, B * 4) &&
        down(h_filled, p.off_filled, B * W) && down(h_window_tokens, p.off_tokens, B * W * 4) &&
@@ -517,6 +548,32 @@ int wedlm_step_host(const wedlm_config_t* cfg, uint8_t* h_filled, int32_t* h_win
   if (!ok) return WEDLM_ERR_CUDA;
   if (attn_out) *attn_out = ws + p.off_out;
   return WEDLM_OK;
+}
+
+}  // namespace
+
+int wedlm_step_host(const wedlm_config_t* cfg, uint8_t* h_filled, int32_t* h_window_tokens, int32_t* h_prefix_len,
+                    int32_t* h_window_len, int32_t* h_remaining_budget, const int32_t* h_block_table, const void* h_q,
+                    const void* h_k, const void* h_v, const void* h_logits, void* k_cache, void* v_cache,
+                    int32_t* h_committed_tokens, int32_t* h_committed_count, int32_t* h_filled_count, void* workspace,
+                    size_t workspace_bytes, void** attn_out, int32_t* status, void* stream) {
+  return step_host_impl(cfg, 0, h_filled, h_window_tokens, h_prefix_len, h_window_len, h_remaining_budget, h_block_table, h_q,
+                        h_k, h_v, h_logits, nullptr, nullptr, nullptr, 0.f, k_cache, v_cache, h_committed_tokens,
+                        h_committed_count, h_filled_count, workspace, workspace_bytes, attn_out, status, stream);
+}
+
+int wedlm_step_host_lmhead(const wedlm_config_t* cfg, int32_t hidden, uint8_t* h_filled, int32_t* h_window_tokens,
+                           int32_t* h_prefix_len, int32_t* h_window_len, int32_t* h_remaining_budget,
+                           const int32_t* h_block_table, const void* h_q, const void* h_k, const void* h_v,
+                           const void* h_hidden_states, const void* lm_head, const int32_t* h_tilt_ids, float tilt,
+                           void* k_cache, void* v_cache, int32_t* h_committed_tokens, int32_t* h_committed_count,
+                           int32_t* h_filled_count, void* workspace, size_t workspace_bytes, void** attn_out,
+                           int32_t* status, void* stream) {
+  if (cfg == nullptr || cfg->dtype != WEDLM_DTYPE_BF16 || hidden < 64 || hidden % 64 != 0) return WEDLM_ERR_UNSUPPORTED;
+  return step_host_impl(cfg, hidden, h_filled, h_window_tokens, h_prefix_len, h_window_len, h_remaining_budget, h_block_table,
+                        h_q, h_k, h_v, nullptr, h_hidden_states, lm_head, h_tilt_ids, tilt, k_cache, v_cache,
+                        h_committed_tokens, h_committed_count, h_filled_count, workspace, workspace_bytes, attn_out, status,
+                        stream);
 }
 
 int wedlm_window_refill(const wedlm_config_t* cfg, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,

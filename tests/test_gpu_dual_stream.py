@@ -119,7 +119,7 @@ def test_fp32_generic_path_small_heads():
         assert err.max() <= 1e-4
 
 
-def test_4k_context_sampled_rows_and_clean_copy_invariant():
+def test_4k_context_every_row_and_clean_copy_invariant():
     c = DS_CONFIGS["ds_4k"]
     inp = make_dual_stream(c, seed=31)
     x, p, im, nobs = _construct(c, inp)
@@ -127,14 +127,22 @@ def test_4k_context_sampled_rows_and_clean_copy_invariant():
     got = _attend(c, inp, p, "auto")
     ph = p.cpu().numpy()
     L = c.seq_len
-    q, k, v, pos = _oracle_inputs(c, inp, 0, ph)
-    g = np.random.default_rng(5)
-    rows = sorted(set(g.integers(0, 2 * L, size=20).tolist()) | {0, L - 1, L, L + 31, L + 32, 2 * L - 1})
-    ref = ds.attention(q, k, v, pos, c.block, theta=c.rope_theta, rows=rows)
-    for a in rows:
-        s, i = divmod(a, L)
-        err = _vec_err(got[0, s, i], ref[a])
-        assert err.max() <= ATTN_REL_TOL, (a, err.max())
+    # Every one of the 2 L rows of every head (262 144 output vectors) against the dense form of the oracle.
+    # The error of a vector is the sum of three bf16 roundings (rotated q, P, the output; typically 3 to 5e-3 of
+    # the vector's largest element) measured against that largest element, which for an average over thousands
+    # of N(0,1) values can itself be small.  Over a quarter of a million vectors the tail of that distribution
+    # reaches past 1e-2 on a few of them (measured: one vector at 1.14e-2), so the criterion here is: at most
+    # one vector in ten thousand above 1e-2, none above 1.5e-2.
+    for n in range(c.n_seq):
+        q, k, v, pos = _oracle_inputs(c, inp, n, ph)
+        ref = ds.attention_dense(q, k, v, pos, c.block, theta=c.rope_theta)
+        err = np.concatenate([_vec_err(got[n, 0, :L], ref[:L]), _vec_err(got[n, 1, :L], ref[L:])])
+        assert np.isfinite(got[n]).all()
+        over = int((err > ATTN_REL_TOL).sum())
+        print("dual-stream 4k: vectors", err.size, "median err", float(np.median(err)), "99.9%", float(np.quantile(err, 0.999)),
+              "max", float(err.max()), "above 1e-2:", over)
+        assert over <= err.size // 10000, (n, over)
+        assert err.max() <= 1.5e-2, (n, np.unravel_index(err.argmax(), err.shape), err.max())
     # nothing masked and the prediction stream a copy of the memory stream: both streams must agree row for row
     inp2 = dict(inp)
     inp2["masked"] = np.zeros_like(inp["masked"])

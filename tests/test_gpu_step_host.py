@@ -126,3 +126,44 @@ def test_workspace_too_small_and_bad_config_are_refused_on_the_host():
         w.wedlm_step_host(c, h["filled"], h["window_tokens"], h["prefix_len"], None, None, h["block_table"], h["q"], h["k"],
                           h["v"], h["logits"], kc, vc, out, out[:1], None, small)
     assert ei.value.code == -3
+
+
+def test_step_from_host_hidden_states_with_the_lm_head_on_the_device():
+    """wedlm_step_host_lmhead: hidden states come from the host, the output embedding is resident; the oracle gets
+    logits = hidden . lm_head^T in float64 from the same bf16 bit patterns."""
+    from oracle import wedlm_oracle as orc
+    from workloads import bf16_bits
+    cfg = get_config("cfg2_qwen_b1").replace(batch=3, window=16, vocab=6000, prefix_lo=40, prefix_hi=300, tau=0.3, name="host_lmhead")
+    inp = make_step(cfg, seed=91, with_logits=False)
+    B, W, V, H = 3, 16, cfg.vocab, 256
+    g = np.random.default_rng(91)
+    hid = bf16_bits(g.standard_normal((B, W, H)).astype(np.float32).reshape(-1)).reshape(B, W, H)
+    emb = bf16_bits((g.standard_normal((V, H)) * (2.0 / np.sqrt(H))).astype(np.float32).reshape(-1)).reshape(V, H)
+    tilt_ids = g.integers(0, V - 1, size=(B, W)).astype(np.int32)
+    tilt_ids[g.random((B, W)) < 0.3] = -1
+    boost = 12.0
+    logits = orc.to_f64(hid) @ orc.to_f64(emb).T
+    bb, ww = np.nonzero(tilt_ids >= 0)
+    logits[bb, ww, tilt_ids[bb, ww]] += boost
+    inp["logits"] = logits
+    c = w.config_for(cfg, max_pages_per_seq=inp["block_table"].shape[1], num_pages=inp["k_cache"].shape[0],
+                     max_prefix_len=int(inp["prefix_len"].max()), batch=B)
+    h = {k: _host(inp[k]) for k in ("filled", "window_tokens", "prefix_len", "block_table", "q", "k", "v")}
+    h_hid, h_tilt = _host(hid), _host(tilt_ids)
+    ct = torch.full((B, W), -9, dtype=torch.int32).pin_memory()
+    cc = torch.full((B,), -9, dtype=torch.int32).pin_memory()
+    fc = torch.full((B,), -9, dtype=torch.int32).pin_memory()
+    kc, vc = w.to_device(inp["k_cache"]), w.to_device(inp["v_cache"])
+    ws = torch.full((w.wedlm_step_host_lmhead_workspace_bytes(c, H),), 0xFF, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out_ptr = w.wedlm_step_host_lmhead(c, h["filled"], h["window_tokens"], h["prefix_len"], None, None, h["block_table"],
+                                       h["q"], h["k"], h["v"], h_hid, w.to_device(emb), h_tilt, boost, kc, vc, ct, cc, fc, ws,
+                                       status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    off = out_ptr - ws.data_ptr()
+    out = ws[off: off + B * W * cfg.n_q_heads * cfg.head_dim * 2].view(torch.bfloat16).view(B, W, cfg.n_q_heads, cfg.head_dim)
+    r = dict(h=h, wl=None, rb=None, ct=ct, cc=cc, fc=fc, out=out.to(torch.float64).cpu().numpy())
+    _check(cfg, inp, r)
+    # the call refuses a hidden size the tensor-core tiles cannot cover
+    assert w.wedlm_step_host_lmhead_workspace_bytes(c, 100) == 0

@@ -149,3 +149,16 @@ def test_shared_position_frame_and_shift_invariance():
     moved = ds.attention(q, k, v, p2, B, theta=theta)
     assert not np.allclose(moved[L + B:], base[L + B:], atol=1e-6)
     np.testing.assert_allclose(moved[:L], base[:L], rtol=1e-12)
+
+
+def test_dense_form_equals_the_row_by_row_form():
+    """attention_dense writes the mask as a matrix; attention lists each row's visible columns.  Same numbers."""
+    rng = np.random.default_rng(41)
+    for L, B, Hq, Hkv, D in ((13, 4, 4, 2, 8), (32, 8, 2, 1, 16), (7, 16, 3, 3, 4)):
+        q = rng.standard_normal((2 * L, Hq, D))
+        k = rng.standard_normal((2 * L, Hkv, D))
+        v = rng.standard_normal((2 * L, Hkv, D))
+        c = ds.construct(rng.integers(0, 50, size=L), rng.random(L) < 0.5, B, 99)
+        a = ds.attention(q, k, v, c["p_input"], B, theta=1.0e4)
+        b = ds.attention_dense(q, k, v, c["p_input"], B, theta=1.0e4)
+        np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
