@@ -280,7 +280,7 @@ def time_workload(wl, steps, warmup, sampler=None, tag="timed", min_region_s=1.0
     block_ms, attn_ms_sum, launches = [], 0.0, 0
     if sampler:
         sampler.tag = tag
-    while sum(block_ms) < min_region_s * 1e3 and len(block_ms) < max_blocks:
+    while not block_ms or (sum(block_ms) < min_region_s * 1e3 and len(block_ms) < max_blocks):
         wl.reset_states()
         l0 = w.wedlm_launch_count()
         start.record()
@@ -328,7 +328,7 @@ def time_graph(wl, steps, warmup, min_region_s=0.25):
     torch.cuda.synchronize()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     total, n = 0.0, 0
-    while total < min_region_s * 1e3 and n < 2000 * steps:
+    while n == 0 or (total < min_region_s * 1e3 and n < 2000 * steps):
         start.record()
         for _ in range(steps):
             graph.replay()
