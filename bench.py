@@ -726,56 +726,67 @@ def run_lmhead(args):
 
 
 def measure_lmhead(steps, warmup):
-    """LM head + confidence/commit at the end-to-end configuration's shape (16 x 16 rows, hidden 4096, vocabulary
-    151 936): the fused call (logits stay in tensor memory) against a library GEMM that writes bf16 logits
-    followed by the streaming confidence call."""
+    """LM head + confidence/commit, hidden 4096 and vocabulary 151 936, at two row counts: 16 x 16 (the shape of a
+    small serving batch) and 64 x 32 (the headline workload's windows, 30 % of the slots already filled).  The fused
+    call (mask rows gathered, logits kept in tensor memory) against a library GEMM over all rows that writes bf16
+    logits followed by the streaming confidence call."""
     import torch
     from paper_2512_22737_b200 import build as b
     b.build()
     import paper_2512_22737_b200 as w
     torch.cuda.set_device(0)
-    B, W, V, H = 16, 16, 151936, 4096
+    V, H = 151936, 4096
     torch.manual_seed(0)
-    hid = torch.randn(B, W, H, device="cuda").to(torch.bfloat16)
     emb = (torch.randn(V, H, device="cuda") * 0.02).to(torch.bfloat16)
     emb_hv = emb.t().contiguous()
-    c = w.make_config(batch=B, window=W, n_q_heads=32, n_kv_heads=8, head_dim=128, max_pages_per_seq=4, num_pages=64,
-                      vocab=V, dtype="bf16", mask_token_id=V - 1, max_prefix_len=16)
-    step = w.DecodeStep(c)
-    filled = (torch.rand(B, W, device="cuda") < 0.3).to(torch.uint8)
-    tok = torch.zeros(B, W, dtype=torch.int32, device="cuda")
-    pl = torch.full((B,), 16, dtype=torch.int32, device="cuda")
-    step.reorder(filled, tok, pl)
-    ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c), dtype=torch.uint8, device="cuda")
+    shapes = {}
+    for B, W in ((16, 16), (64, 32)):
+        hid = torch.randn(B, W, H, device="cuda").to(torch.bfloat16)
+        c = w.make_config(batch=B, window=W, n_q_heads=32, n_kv_heads=8, head_dim=128, max_pages_per_seq=4, num_pages=64,
+                          vocab=V, dtype="bf16", mask_token_id=V - 1, max_prefix_len=16)
+        step = w.DecodeStep(c)
+        filled = (torch.rand(B, W, device="cuda") < 0.3).to(torch.uint8)
+        tok = torch.zeros(B, W, dtype=torch.int32, device="cuda")
+        pl = torch.full((B,), 16, dtype=torch.int32, device="cuda")
+        step.reorder(filled, tok, pl)
+        mask_rows = int(B * W - step.n_filled.sum().item())
+        ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c, H), dtype=torch.uint8, device="cuda")
 
-    def fused(f, t, p):
-        w.wedlm_lmhead_confidence_commit(c, hid, emb, None, 0.0, step.perm, step.n_filled, step.n_commit, t, f, p, None, None,
-                                         step.argmax, step.maxprob, step.entropy, step.lse, step.committed_tokens,
-                                         step.committed_count, step.filled_count, ws)
+        def fused(f, t, p):
+            w.wedlm_lmhead_confidence_commit(c, hid, emb, None, 0.0, step.perm, step.n_filled, step.n_commit, t, f, p, None,
+                                             None, step.argmax, step.maxprob, step.entropy, step.lse, step.committed_tokens,
+                                             step.committed_count, step.filled_count, ws, step.status)
 
-    def unfused(f, t, p):
-        step.confidence_commit((hid @ emb_hv).contiguous(), t, f, p)
+        def unfused(f, t, p):
+            step.confidence_commit((hid @ emb_hv).contiguous(), t, f, p)
 
-    out = {}
-    for name, fn in (("fused", fused), ("gemm_then_confidence", unfused)):
-        ts = []
-        for _ in range(warmup + steps):
-            f, t, p = filled.clone(), tok.clone(), pl.clone()
-            a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            fn(f, t, p)
-            e.record()
-            torch.cuda.synchronize()
-            ts.append(a.elapsed_time(e))
-        ts = ts[warmup:]
-        out[name] = {"ms_min": min(ts), "ms_median": statistics.median(ts)}
-    weights = V * H * 2
-    line = {"metric": "lm_head_confidence_ms", "unit": "ms", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "lmhead", "rows": B * W, "hidden": H, "vocab": V},
-            "results": out, "weight_bytes": weights, "flops": 2 * B * W * H * V,
-            "fused_weight_stream_GBps": weights / (out["fused"]["ms_median"] * 1e-3) / 1e9,
-            "fused_TFLOPs": 2 * B * W * H * V / (out["fused"]["ms_median"] * 1e-3) / 1e12}
-    return line
+        out = {}
+        for name, fn in (("fused", fused), ("gemm_then_confidence", unfused)):
+            ts = []
+            for _ in range(warmup + steps):
+                f, t, p = filled.clone(), tok.clone(), pl.clone()
+                a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn(f, t, p)
+                e.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(e))
+            ts = ts[warmup:]
+            out[name] = {"ms_min": min(ts), "ms_median": statistics.median(ts)}
+        assert int(step.status.item()) == 0
+        # the tensor cores run whole 256-row chunks of the gathered mask rows; the flops that count are the mask rows'
+        chunks = (mask_rows + 255) // 256
+        t = out["fused"]["ms_median"] * 1e-3
+        out.update({"rows": B * W, "mask_rows": mask_rows, "flops_mask_rows": 2 * mask_rows * H * V,
+                    "flops_tiles": 2 * chunks * 256 * H * V,
+                    "fused_TFLOPs_mask_rows": 2 * mask_rows * H * V / t / 1e12,
+                    "fused_TFLOPs_tiles": 2 * chunks * 256 * H * V / t / 1e12,
+                    "fused_weight_stream_GBps": V * H * 2 / t / 1e9})
+        shapes[f"{B}x{W}"] = out
+        del hid, ws, step
+    return {"metric": "lm_head_confidence_ms", "unit": "ms", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "lmhead", "hidden": H, "vocab": V, "filled_fraction": 0.3},
+            "weight_bytes": V * H * 2, "shapes": shapes}
 
 
 # ----------------------------------------------------------------------------------------------

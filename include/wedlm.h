@@ -255,10 +255,14 @@ int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const
  *   all other arguments as in wedlm_confidence_commit; statistics come from fp32 logits (not rounded to bf16).
  *   cfg->sample_temperature must be 0 (the logits are never stored, so there is nothing to draw from after the
  *   selection): WEDLM_ERR_UNSUPPORTED otherwise.
- * Workspace: wedlm_lmhead_confidence_workspace_bytes(cfg) = batch*window*ceil(vocab/128)*16 bytes (an upper
- * bound: the vocabulary tile width, 128..256, is chosen per launch).
+ * Only the mask rows get logits (Algorithm 1 predicts from l_mask): their hidden states are first gathered into a
+ * dense matrix inside the workspace, so the tensor-core tiles hold nothing but rows that count.
+ * Workspace: wedlm_lmhead_confidence_workspace_bytes(cfg, hidden) bytes = the chunk partials
+ * (batch*window*ceil(vocab/128)*16, an upper bound: the vocabulary tile width, 128..256, is chosen per launch), the
+ * row map and the gathered hidden states (batch*window*hidden*2).
+ *   status        in/out i32 [1] or NULL; WEDLM_STATUS_WAIT_EXPIRED if a bounded on-chip wait gave up
  */
-size_t wedlm_lmhead_confidence_workspace_bytes(const wedlm_config_t* cfg);
+size_t wedlm_lmhead_confidence_workspace_bytes(const wedlm_config_t* cfg, int32_t hidden);
 int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, const void* hidden_states,
                                    const void* lm_head, const int32_t* tilt_ids, float tilt,
                                    const int32_t* perm, const int32_t* n_filled, const int32_t* n_commit,

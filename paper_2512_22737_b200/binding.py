@@ -94,7 +94,7 @@ def load_library() -> ctypes.CDLL:
     lib.wedlm_confidence_commit_static.argtypes = [cfgp, vp, i32p, i32p, i32p, i32p, u8p, i32p, i32p, i32p,
                                                    i32p, f32p, f32p, f32p, i32p, i32p, i32p, i32p, vp]
     lib.wedlm_lmhead_confidence_workspace_bytes.restype = ctypes.c_size_t
-    lib.wedlm_lmhead_confidence_workspace_bytes.argtypes = [cfgp]
+    lib.wedlm_lmhead_confidence_workspace_bytes.argtypes = [cfgp, ctypes.c_int32]
     lib.wedlm_lmhead_confidence_commit.restype = ctypes.c_int
     lib.wedlm_lmhead_confidence_commit.argtypes = [cfgp, ctypes.c_int32, vp, vp, i32p, ctypes.c_float, i32p, i32p, i32p,
                                                    i32p, u8p, i32p, i32p, i32p, i32p, f32p, f32p, f32p, i32p, i32p,
@@ -251,8 +251,8 @@ def wedlm_confidence_commit(cfg, logits, perm, n_filled, n_commit, window_tokens
         _ptr(status, i32, "status"), _stream(stream)), "wedlm_confidence_commit")
 
 
-def wedlm_lmhead_confidence_workspace_bytes(cfg) -> int:
-    return int(load_library().wedlm_lmhead_confidence_workspace_bytes(ctypes.byref(cfg)))
+def wedlm_lmhead_confidence_workspace_bytes(cfg, hidden: int) -> int:
+    return int(load_library().wedlm_lmhead_confidence_workspace_bytes(ctypes.byref(cfg), ctypes.c_int32(hidden)))
 
 
 def wedlm_lmhead_confidence_commit(cfg, hidden_states, lm_head, tilt_ids, tilt, perm, n_filled, n_commit, window_tokens,

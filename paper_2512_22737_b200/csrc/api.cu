@@ -262,10 +262,9 @@ int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const
                            committed_count, filled_count, workspace, status, (cudaStream_t)stream);
 }
 
-size_t wedlm_lmhead_confidence_workspace_bytes(const wedlm_config_t* cfg) {
-  if (check_config(cfg, false, true) != WEDLM_OK) return 0;
-  size_t b = (size_t)cfg->batch * cfg->window * lmhead_conf_tiles(cfg->vocab) * 16;
-  return b ? b : 256;
+size_t wedlm_lmhead_confidence_workspace_bytes(const wedlm_config_t* cfg, int32_t hidden) {
+  if (check_config(cfg, false, true) != WEDLM_OK || hidden < 64 || hidden % 64 != 0) return 0;
+  return lmhead_workspace(cfg, hidden).total;
 }
 
 int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, const void* hidden_states,
@@ -284,11 +283,12 @@ int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, co
   if (!hidden_states || !lm_head || !perm || !n_filled || !n_commit || !window_tokens || !filled || !prefix_len || !workspace)
     return WEDLM_ERR_INVALID_ARG;
   if (!aligned16(hidden_states) || !aligned16(lm_head) || !aligned16(workspace)) return WEDLM_ERR_INVALID_ARG;
-  if (workspace_bytes < wedlm_lmhead_confidence_workspace_bytes(cfg)) return WEDLM_ERR_WORKSPACE_TOO_SMALL;
+  const LmWorkspace lw = lmhead_workspace(cfg, hidden);
+  if (workspace_bytes < lw.total) return WEDLM_ERR_WORKSPACE_TOO_SMALL;
   Shape s = make_shape(cfg);
   cudaStream_t st = (cudaStream_t)stream;
   int n_tiles = 0;
-  rc = launch_lmhead_conf(s, hidden, hidden_states, lm_head, tilt_ids, tilt, n_filled, window_len, workspace, &n_tiles, status, st);
+  rc = launch_lmhead_conf(s, hidden, hidden_states, lm_head, tilt_ids, tilt, n_filled, window_len, workspace, lw, &n_tiles, status, st);
   if (rc != WEDLM_OK) return rc;
   return launch_conf_commit(s, cfg, n_tiles, workspace, perm, n_filled, n_commit, window_tokens, filled,
                             prefix_len, window_len, remaining_budget, argmax, maxprob, entropy, lse, committed_tokens,
@@ -426,7 +426,7 @@ int plan_host_step(const wedlm_config_t* cfg, int32_t hidden, HostStepPlan* out)
   p.off_ccount = take(B * 4);
   p.off_fcount = take(B * 4);
   p.attn_ws_bytes = plan_attention(cfg).total_bytes;
-  p.conf_ws_bytes = hidden > 0 ? wedlm_lmhead_confidence_workspace_bytes(cfg) : confidence_workspace_bytes(cfg);
+  p.conf_ws_bytes = hidden > 0 ? wedlm_lmhead_confidence_workspace_bytes(cfg, hidden) : confidence_workspace_bytes(cfg);
   p.off_attn_ws = take(p.attn_ws_bytes);
   p.off_conf_ws = take(p.conf_ws_bytes);
   p.total = at;

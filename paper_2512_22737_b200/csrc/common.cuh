@@ -106,11 +106,16 @@ int launch_conf_commit(const Shape& s, const wedlm_config_t* cfg, int n_chunks, 
                        float* maxprob, float* entropy, float* lse, int32_t* committed_tokens, int32_t* committed_count,
                        int32_t* filled_count, cudaStream_t st, void* sample_ws = nullptr);
 
-// Fused LM head + confidence pass 1: partials [B*W][n_tiles] (n_tiles <= ceil(V/128), returned) from hidden states and the output embedding.
+// Fused LM head + confidence pass 1: partials [B*W][n_tiles] (n_tiles <= ceil(V/128), returned) from hidden states and the
+// output embedding.  Only the mask rows are computed: they are gathered into a dense matrix in the workspace first.
+struct LmWorkspace {
+  size_t off_part, off_count, off_map, off_dense, total;
+};
 int lmhead_conf_tiles(int vocab);
+LmWorkspace lmhead_workspace(const wedlm_config_t* cfg, int hidden);
 int launch_lmhead_conf(const Shape& s, int hidden, const void* hidden_states, const void* lm_head, const int32_t* tilt_ids,
-                       float tilt, const int32_t* n_filled, const int32_t* window_len, void* partials, int* n_tiles_out,
-                       int32_t* status, cudaStream_t st);
+                       float tilt, const int32_t* n_filled, const int32_t* window_len, void* workspace,
+                       const LmWorkspace& lw, int* n_tiles_out, int32_t* status, cudaStream_t st);
 
 // Dual-Stream Masking (training forward): input construction and the per-unit page tables.
 int launch_dual_stream_construct(int N, int L, int B, int K, int mask_id, const int32_t* tokens, const uint8_t* masked,

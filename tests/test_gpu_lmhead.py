@@ -10,13 +10,17 @@ from workloads import StepConfig, bf16_bits, make_step
 pytestmark = pytest.mark.gpu
 
 
-def _case(B, W, V, H, seed, boost=6.0, window_len=None, budget=None, commit_mode="streaming"):
+def _case(B, W, V, H, seed, boost=6.0, window_len=None, budget=None, commit_mode="streaming", fill_all=()):
     import paper_2512_22737_b200 as w
     import parity_util as pu
     cfg = StepConfig(name="lmhead", batch=B, window=W, n_q_heads=4, n_kv_heads=1, head_dim=128, vocab=V, dtype="bf16",
                      prefix_lo=10, prefix_hi=60, obs_prob_lo=0.2, obs_prob_hi=0.6, tau=0.3, lam=0.1)
     inp = make_step(cfg, seed=seed, with_logits=False)
     g = np.random.default_rng(seed)
+    if len(fill_all):                                    # sequences without a single mask row
+        f = inp["filled"].copy()
+        f[list(fill_all)] = 1
+        inp = make_step(cfg, seed=seed, with_logits=False, filled=f)
     hid = bf16_bits((g.standard_normal((B, W, H)) * 1.0).astype(np.float32).reshape(-1)).reshape(B, W, H)
     emb = bf16_bits((g.standard_normal((V, H)) * (2.0 / np.sqrt(H))).astype(np.float32).reshape(-1)).reshape(V, H)
     tilt_ids = g.integers(0, V - 1, size=(B, W)).astype(np.int32)
@@ -36,7 +40,7 @@ def _case(B, W, V, H, seed, boost=6.0, window_len=None, budget=None, commit_mode
     wl = None if window_len is None else torch.tensor(window_len, dtype=torch.int32, device="cuda")
     bud = None if budget is None else torch.tensor(budget, dtype=torch.int32, device="cuda")
     step.reorder(d["filled"], d["window_tokens"], d["prefix_len"], wl)
-    ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c, H), dtype=torch.uint8, device="cuda")
     w.wedlm_lmhead_confidence_commit(c, w.to_device(hid), w.to_device(emb), w.to_device(tilt_ids), boost, step.perm,
                                      step.n_filled, step.n_commit, d["window_tokens"], d["filled"], d["prefix_len"], wl, bud,
                                      step.argmax, step.maxprob, step.entropy, step.lse, step.committed_tokens,
@@ -69,6 +73,18 @@ def test_fused_lmhead_confidence_matches_oracle(B, W, V, H):
 def test_fused_lmhead_short_windows_budget_and_block_mode():
     _case(4, 8, 2048, 128, seed=9, window_len=[8, 5, 3, 8], budget=[10, 1, 0, 10])
     _case(4, 8, 2048, 128, seed=10, commit_mode="block")
+
+
+def test_fused_lmhead_sequences_without_mask_rows_and_a_batch_without_any():
+    """The mask rows are gathered before the tensor-core pass: sequences that contribute none, and a call in which
+    no row at all is a mask (the pass runs over zero items and only the commit/shift part does anything)."""
+    _case(4, 8, 2048, 128, seed=21, fill_all=(0, 2))
+    _case(3, 8, 2048, 128, seed=22, fill_all=(0, 1, 2))
+
+
+def test_fused_lmhead_more_sequences_than_one_scan_pass():
+    """1100 sequences: the per-sequence mask-row counts are scanned 1024 at a time with a carry."""
+    _case(1100, 4, 512, 64, seed=23)
 
 
 def test_fused_lmhead_qwen_width_rows_over_256():
@@ -104,7 +120,7 @@ def test_tile_width_that_is_no_multiple_of_32_ignores_stale_tensor_memory():
     big = torch.full((B, W, H), 1.0e19, dtype=torch.bfloat16, device="cuda")
     emb1 = torch.full((V1, H), 1.0e19, dtype=torch.bfloat16, device="cuda")
     s1.reorder(filled, tok, pl)
-    ws1 = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c1), dtype=torch.uint8, device="cuda")
+    ws1 = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c1, H), dtype=torch.uint8, device="cuda")
     w.wedlm_lmhead_confidence_commit(c1, big, emb1, None, 0.0, s1.perm, s1.n_filled, s1.n_commit, tok.clone(), filled.clone(),
                                      pl.clone(), None, None, s1.argmax, s1.maxprob, s1.entropy, s1.lse, s1.committed_tokens,
                                      s1.committed_count, s1.filled_count, ws1)

@@ -167,7 +167,7 @@ def test_fused_lm_head_refuses_sampling_and_workspace_grows():
     fil = torch.zeros(B, W, dtype=torch.uint8, device="cuda")
     pl = torch.zeros(B, **i32)
     s.reorder(fil, tok, pl)
-    ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c1), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(c1, H), dtype=torch.uint8, device="cuda")
     with pytest.raises(w.WedlmError) as ei:
         w.wedlm_lmhead_confidence_commit(c1, hs, emb, None, 0.0, s.perm, s.n_filled, s.n_commit, tok, fil, pl, None, None,
                                          s.argmax, s.maxprob, s.entropy, s.lse, s.committed_tokens, s.committed_count,
