@@ -17,7 +17,8 @@
 // tcgen05.commit, warps 0-7 read their row of the accumulators back with tcgen05.ld and reduce it.  The wide tile
 // matters: every item re-reads the hidden states from L2, and with tiles of 128 (two accumulator sets, reduction
 // overlapped with the next item's MMAs) the extra L2 traffic cost more than the overlap won.  Requesting the
-// embedding tiles into L2 ahead of the ring did not help either.  All waits are bounded.
+// embedding tiles into L2 ahead of the ring, or giving them a deeper ring of their own (5 stages beside 3 for the
+// hidden states), made the kernel slower; a 2-stage ring costs 22 %.  All waits are bounded.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include <math_constants.h>
@@ -32,10 +33,7 @@ using namespace ptx;
 
 constexpr int kLmMaxTileN = 256;              // most vocabulary entries per work item (the host picks 128..256)
 constexpr int kLmTileK = 64;                  // hidden elements per stage (one 128-byte swizzle row)
-#ifndef WEDLM_LM_STAGES
-#define WEDLM_LM_STAGES 3
-#endif
-constexpr int kLmStages = WEDLM_LM_STAGES;
+constexpr int kLmStages = 3;
 constexpr int kLmRows = 256;                  // window rows per work item (two 128-row accumulators)
 constexpr uint32_t kLmBytesA = 128 * 128;     // one 128-row tile of hidden states per stage
 constexpr uint32_t kLmStrideB = kLmMaxTileN * 128;               // room of the embedding tile per stage
