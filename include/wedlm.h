@@ -27,10 +27,13 @@
  *   - No result of one call is remembered for the next.  What the library does keep per process is
  *     bookkeeping only: a count of the kernels it launched (wedlm_launch_count), the one-shot timing
  *     hook armed by wedlm_profile_next_attn (per host thread), per-device attributes it asked the
- *     driver for once (SM count, shared-memory opt-ins) and the device address of the built-in
- *     scratch array.
+ *     driver for once (SM count, shared-memory opt-ins), the device address of the built-in
+ *     scratch array, and the copy stream with its two events that the wedlm_step_host calls use
+ *     (per host thread and device, created on first use).
  *   - Calls are asynchronous on the CUDA stream passed as `stream` (a cudaStream_t cast to
- *     void*; NULL is the legacy default stream).  No call synchronises with the host.
+ *     void*; NULL is the legacy default stream).  No call synchronises with the host.  The
+ *     wedlm_step_host calls fork their large upload onto a copy stream of the library and join it
+ *     back into `stream` before they return: to the caller everything is ordered on `stream`.
  *   - All tensors are dense, row-major ("last index fastest") and need 16-byte aligned base
  *     addresses.  Index tensors are int32, flags are uint8.
  *   - "logical order" = ascending position id within the window; "physical order" = the order
@@ -322,8 +325,10 @@ int wedlm_window_refill(const wedlm_config_t* cfg, const int32_t* n_commit,
  * One whole step of Algorithm 1 (reorder -> window attention -> confidence / commit / refill) for callers whose
  * step inputs live in HOST memory.  The call enqueues, on `stream`: the host-to-device copies of the inputs into
  * `workspace`, the kernels of wedlm_reorder, wedlm_window_attn and wedlm_confidence_commit, and the device-to-host
- * copies of the results; it returns without waiting (synchronise the stream before reading the outputs).  Use
- * page-locked host memory, or the copies serialise with the host.
+ * copies of the results; it returns without waiting (synchronise the stream before reading the outputs).  The largest
+ * upload (logits, or hidden states) travels on a copy stream of the library while reorder and attention run, and is
+ * joined back into `stream` in front of the confidence pass.  Use page-locked host memory, or the copies serialise
+ * with the host.
  *   h_filled, h_window_tokens, h_prefix_len   host, in/out: the window state, updated in place by the step
  *   h_window_len, h_remaining_budget          host, in/out, each may be NULL (meaning as in wedlm_confidence_commit)
  *   h_block_table, h_q, h_k, h_v, h_logits    host, in: layouts as in wedlm_window_attn / wedlm_confidence_commit.

@@ -450,6 +450,29 @@ size_t wedlm_step_host_lmhead_workspace_bytes(const wedlm_config_t* cfg, int32_t
 
 namespace {
 
+// The large upload of a host step (hidden states or logits) runs on a copy stream of its own, forked from and joined
+// back into the caller's stream with two events, so that it overlaps the reorder / RoPE / attention kernels instead
+// of queueing behind them.  One lane per host thread and device, created on first use and kept.
+struct CopyLane {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+  bool ready = false;
+};
+
+CopyLane* copy_lane() {
+  thread_local CopyLane lanes[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  CopyLane& l = lanes[dev];
+  if (!l.ready) {
+    if (cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&l.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&l.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    l.ready = true;
+  }
+  return &l;
+}
+
 // Both host-step calls: logits from the host (h_hidden == NULL) or hidden states from the host with the output
 // embedding resident on the device.
 int step_host_impl(const wedlm_config_t* cfg, int32_t hidden, uint8_t* h_filled, int32_t* h_window_tokens,
@@ -487,6 +510,50 @@ int step_host_impl(const wedlm_config_t* cfg, int32_t hidden, uint8_t* h_filled,
   if (ok && h_window_len) ok = up(p.off_wlen, h_window_len, B * 4);
   if (ok && h_remaining_budget) ok = up(p.off_budget, h_remaining_budget, B * 4);
   if (!ok) return WEDLM_ERR_CUDA;
+  // The copy lane starts after the uploads above (the copy engine serves them first: the kernels need them first)
+  // and after whatever the caller's stream still had queued on this workspace.
+  CopyLane* lane = copy_lane();
+  if (!lane) return WEDLM_ERR_CUDA;
+  if (cudaEventRecord(lane->fork, st) != cudaSuccess || cudaStreamWaitEvent(lane->stream, lane->fork, 0) != cudaSuccess)
+    return WEDLM_ERR_CUDA;
+  auto up_lane = [&](size_t off, const void* src, size_t bytes) {
+    return cudaMemcpyAsync(ws + off, src, bytes, cudaMemcpyHostToDevice, lane->stream) == cudaSuccess;
+  };
+  // Whatever happens from here on, the lane is joined back into the caller's stream before this call returns: in
+  // front of the confidence pass when all goes well, on the way out otherwise.
+  struct Join {
+    cudaStream_t st;
+    CopyLane* lane;
+    bool recorded = false, waited = false;
+    bool wait() {
+      if (waited || !recorded) return true;
+      waited = true;
+      return cudaStreamWaitEvent(st, lane->join, 0) == cudaSuccess;
+    }
+    ~Join() { wait(); }
+  } join{st, lane};
+  bool big_ok = true;
+  if (fused) {
+    // hidden states of all rows (the mask rows are gathered on the device), tilt ids if any
+    big_ok = up_lane(p.off_logits, h_hidden, B * W * (size_t)hidden * elem);
+    if (big_ok && h_tilt_ids) big_ok = up_lane(p.off_tilt, h_tilt_ids, B * W * 4);
+  } else {
+    // Logits: only the rows the confidence pass reads.  After reordering the mask rows of a sequence are the
+    // physical rows [n_filled, window_len), one contiguous range, and n_filled is a count over the host's flags.
+    for (size_t b = 0; big_ok && b < B; ++b) {
+      long long L = h_window_len ? h_window_len[b] : (long long)W;
+      L = L < 0 ? 0 : (L > (long long)W ? (long long)W : L);
+      long long nf = 0;
+      for (long long j = 0; j < L; ++j) nf += h_filled[b * W + j] != 0;
+      if (L > nf) {
+        const size_t off = (b * W + (size_t)nf) * (size_t)cfg->vocab * elem;
+        big_ok = up_lane(p.off_logits + off, static_cast<const char*>(h_logits) + off, (size_t)(L - nf) * cfg->vocab * elem);
+      }
+    }
+  }
+  if (cudaEventRecord(lane->join, lane->stream) != cudaSuccess) return WEDLM_ERR_CUDA;
+  join.recorded = true;
+  if (!big_ok) return WEDLM_ERR_CUDA;
   uint8_t* d_filled = reinterpret_cast<uint8_t*>(ws + p.off_filled);
   int32_t* d_tokens = reinterpret_cast<int32_t*>(ws + p.off_tokens);
   int32_t* d_prefix = reinterpret_cast<int32_t*>(ws + p.off_prefix);
@@ -511,29 +578,14 @@ int step_host_impl(const wedlm_config_t* cfg, int32_t hidden, uint8_t* h_filled,
   int32_t* d_ctok = reinterpret_cast<int32_t*>(ws + p.off_ctok);
   int32_t* d_ccount = reinterpret_cast<int32_t*>(ws + p.off_ccount);
   int32_t* d_fcount = reinterpret_cast<int32_t*>(ws + p.off_fcount);
+  if (!join.wait()) return WEDLM_ERR_CUDA;             // the hidden states / logits have landed
   if (fused) {
-    // hidden states of all rows (the tensor-core tiles span whole row blocks), tilt ids if any
-    if (!up(p.off_logits, h_hidden, B * W * (size_t)hidden * elem)) return WEDLM_ERR_CUDA;
-    if (h_tilt_ids && !up(p.off_tilt, h_tilt_ids, B * W * 4)) return WEDLM_ERR_CUDA;
     rc = wedlm_lmhead_confidence_commit(cfg, hidden, ws + p.off_logits, lm_head,
                                         h_tilt_ids ? reinterpret_cast<int32_t*>(ws + p.off_tilt) : nullptr, tilt, d_perm,
                                         d_nfilled, d_ncommit, d_tokens, d_filled, d_prefix, d_wlen, d_budget, d_argmax,
                                         d_maxprob, d_entropy, d_lse, d_ctok, d_ccount, d_fcount, ws + p.off_conf_ws,
                                         p.conf_ws_bytes, status, stream);
   } else {
-    // Logits: only the rows the confidence pass reads.  After reordering the mask rows of a sequence are the
-    // physical rows [n_filled, window_len), one contiguous range, and n_filled is a count over the host's flags.
-    for (size_t b = 0; b < B; ++b) {
-      long long L = h_window_len ? h_window_len[b] : (long long)W;
-      L = L < 0 ? 0 : (L > (long long)W ? (long long)W : L);
-      long long nf = 0;
-      for (long long j = 0; j < L; ++j) nf += h_filled[b * W + j] != 0;
-      if (L > nf) {
-        const size_t off = (b * W + (size_t)nf) * (size_t)cfg->vocab * elem;
-        if (!up(p.off_logits + off, static_cast<const char*>(h_logits) + off, (size_t)(L - nf) * cfg->vocab * elem))
-          return WEDLM_ERR_CUDA;
-      }
-    }
     rc = wedlm_confidence_commit(cfg, ws + p.off_logits, d_perm, d_nfilled, d_ncommit, d_tokens, d_filled, d_prefix, d_wlen,
                                  d_budget, d_argmax, d_maxprob, d_entropy, d_lse, d_ctok, d_ccount, d_fcount,
                                  ws + p.off_conf_ws, p.conf_ws_bytes, status, stream);
