@@ -498,8 +498,8 @@ def run_product(args):
     for mode, r in e2e.items():
         r = r or (float("nan"), 0, 0, 0)
         (e_ms,), (e_commit,) = reduce_over_ranks([r[0]], [r[1]], "cuda")
-        e2e_json[mode] = {"value": (e_commit / (e_ms * 1e-3)) if e_ms == e_ms else None, "unit": UNIT, "ms_per_step": e_ms,
-                          "h2d_bytes_per_step": r[2], "d2h_bytes_per_step": r[3]}
+        e2e_json[mode] = {"value": (e_commit / (e_ms * 1e-3)) if e_ms == e_ms else None, "unit": UNIT,
+                          "ms_per_step": e_ms if e_ms == e_ms else None, "h2d_bytes_per_step": r[2], "d2h_bytes_per_step": r[3]}
     e2e_json["lmhead"]["call"] = "wedlm_step_host_lmhead: hidden states [B,W,4096] from pinned host memory, output embedding resident"
     e2e_json["logits"]["call"] = "wedlm_step_host: logits rows of the mask slots from pinned host memory"
 
@@ -685,21 +685,26 @@ def measure_loop(args):
     lm_head_vh = wts["lm_head"].t().contiguous() if args.loop_fused_windows else None
     for W, mode, fused in runs:
         for tilt_name, tilt in args.loop_tilts:
-            dec = StreamingDecoder(m, {}, batch=B, window=W, max_total_len=P + N, tau=args.loop_tau, lam=args.loop_lambda,
-                                   tilt=0.0, target=pt["target"], commit_mode=mode, fused_lm_head=fused)
-            dec.wt = wts
-            dec.lm_head_vh = lm_head_vh
-            dec.prefill(pt["prompt"])
-            if lse0 is None:                    # log-sum-exp of the untilted logits, measured once
-                dec.start(N)
-                lg, _ = dec.forward()
-                lse0 = float(torch.logsumexp(lg[:, 0].float(), dim=-1).mean().item())
-            dec.tilt = tilt if tilt_name == "literal" else lse0 + tilt
-            torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            out = dec.generate(N, use_graph=not args.loop_eager)
-            torch.cuda.synchronize()
-            dt = time.perf_counter() - t0
+            # a short untimed run of the same geometry first: the first GEMMs of a new shape and the first capture
+            # pay one-off library set-up that is no part of the decode rate
+            for phase_tokens in (min(8, N), N):
+                dec = StreamingDecoder(m, {}, batch=B, window=W, max_total_len=P + N, tau=args.loop_tau, lam=args.loop_lambda,
+                                       tilt=0.0, target=pt["target"], commit_mode=mode, fused_lm_head=fused)
+                dec.wt = wts
+                dec.lm_head_vh = lm_head_vh
+                dec.prefill(pt["prompt"])
+                if lse0 is None:                    # log-sum-exp of the untilted logits, measured once
+                    dec.start(N)
+                    lg, _ = dec.forward()
+                    lse0 = float(torch.logsumexp(lg[:, 0].float(), dim=-1).mean().item())
+                dec.tilt = tilt if tilt_name == "literal" else lse0 + tilt
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                out = dec.generate(phase_tokens, use_graph=not args.loop_eager)
+                torch.cuda.synchronize()
+                dt = time.perf_counter() - t0
+                if phase_tokens != N:
+                    del dec
             n_gen = sum(len(y) for y in out["y"])
             on_target = sum(int(out["y"][bb] == pt["target"][bb, P:P + N].tolist()) for bb in range(B))
             results.append({"window": W, "commit": mode, "lm_head": "fused" if fused else "gemm+logits",
@@ -714,7 +719,7 @@ def measure_loop(args):
             "config": {"workload": "cfg5_loop", "batch": B, "prompt": P, "new_tokens": N, "layers": m.n_layers,
                        "tau": args.loop_tau, "lambda": args.loop_lambda,
                        "hidden": H, "lse_of_untilted_logits": lse0,
-                       "timing": "host wall clock around generate(), includes the graph capture and the per-step read-back of commits"},
+                       "timing": "host wall clock around generate(), after one short untimed run of the same geometry; includes the graph capture and the per-step read-back of commits"},
             "results": results}
     del wts, lm_head_vh
     return line
