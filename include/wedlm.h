@@ -153,7 +153,11 @@ int wedlm_reorder(const wedlm_config_t* cfg, const uint8_t* filled, const int32_
                   int32_t* n_filled, int32_t* n_commit, void* stream);
 
 /* Bytes of workspace wedlm_window_attn needs for this config (uses batch, window, heads,
- * head_dim, dtype, max_prefix_len, attn_impl).  Returns 0 on an invalid config. */
+ * head_dim, dtype, max_prefix_len, attn_impl, and the SM count of the current device).  It holds the
+ * rotated queries and, when the batch has fewer work units than the GPU has CTA slots, room for the
+ * partial results of keys that are split between CTAs (up to about 2*SMs/Hkv pieces per query row,
+ * so a single long sequence can use the whole GPU); only the part that a launch uses is touched.
+ * Returns 0 on an invalid config. */
 size_t wedlm_window_attn_workspace_bytes(const wedlm_config_t* cfg);
 
 /*

@@ -90,31 +90,26 @@ AttnPlan plan_attention(const wedlm_config_t* c) {
   p.impl = (c->attn_impl == WEDLM_ATTN_GENERIC || !tensor_ok) ? WEDLM_ATTN_GENERIC : WEDLM_ATTN_TENSOR;
   long long S, chunk;
   if (p.impl == WEDLM_ATTN_TENSOR) {
-    // one CTA per (sequence, kv head, 128-row tile, key chunk); two CTAs per SM.  Split the keys
-    // only as far as needed to give every CTA slot a few work items; chunks are whole 64-key tiles.
+    // Two CTAs per SM.  With at least one work unit (sequence, kv head, 128-row tile) per CTA slot, every CTA takes
+    // one whole unit, longest first, and no partials exist at all.  With fewer units the 64-key tiles of all units
+    // are cut into one equal run per slot; a unit that is cut leaves one partial per piece, at most n_splits of them
+    // (the kernel keeps its runs long enough for that).
     const int G = c->n_q_heads / c->n_kv_heads;
     const long long w_t = 128 / G;
-    const long long units = (long long)c->batch * c->n_kv_heads * ((c->window + w_t - 1) / w_t);
-    // Sequences are dispatched longest first, so a batch with at least one work unit per CTA slot
-    // (2 per SM) balances well without splitting the keys, and then no partials exist at all.  With
-    // fewer units the keys are split just far enough to fill the slots: the smallest split count
-    // whose last wave is at least 85 % full, chunks no shorter than 256 keys.
+    const long long n_mtiles = (c->window + w_t - 1) / w_t;
+    const long long units = (long long)c->batch * c->n_kv_heads * n_mtiles;
     const long long slots = 2LL * device_sm_count();
-    long long cap = total / 256 > 1 ? total / 256 : 1;
-    if (cap > 64) cap = 64;
     S = 1;
+    chunk = (total + 63) / 64 * 64;
     if (units > 0 && units < slots) {
-      double best = 0.0;
-      for (long long cand = 1; cand <= cap; ++cand) {
-        const long long ctas = units * cand;
-        const long long waves = (ctas + slots - 1) / slots;
-        const double eff = (double)ctas / (double)(waves * slots);
-        if (eff > best + 1e-9) { best = eff; S = cand; }
-        if (eff >= 0.85) { S = cand; break; }
-      }
+      p.balanced = 1;
+      const long long n_runs = slots / n_mtiles > 0 ? slots / n_mtiles : 1;     // a run is shared by the row tiles
+      p.n_ctas = (int)(n_runs * n_mtiles);
+      const long long t_max = (total + 63) / 64;
+      S = n_runs / c->n_kv_heads + 3;
+      if (S > t_max) S = t_max;
+      if (S < 2) S = 2;
     }
-    chunk = (total + S - 1) / S;
-    chunk = (chunk + 63) / 64 * 64;
   } else {
     const long long n_rb = (c->window + 15) / 16;
     const long long units = (long long)c->batch * c->n_q_heads * n_rb;
@@ -124,7 +119,7 @@ AttnPlan plan_attention(const wedlm_config_t* c) {
     chunk = (total + S - 1) / S;
     chunk = (chunk + c->page_size - 1) / c->page_size * c->page_size;
   }
-  S = (total + chunk - 1) / chunk;
+  if (!p.balanced) S = (total + chunk - 1) / chunk;
   p.n_splits = (int)S;
   p.chunk = (int)chunk;
   p.q_rot_bytes = align_up((size_t)c->batch * c->window * c->n_q_heads * c->head_dim * elem, 256);
@@ -133,7 +128,8 @@ AttnPlan plan_attention(const wedlm_config_t* c) {
     p.part_o_bytes = align_up(rows * c->head_dim * sizeof(float), 256);
     p.part_ml_bytes = align_up(rows * 2 * sizeof(float), 256);
   }
-  p.order_bytes = align_up((size_t)c->batch * sizeof(int32_t), 256);
+  // dispatch order of the sequences (i32 per sequence), or the record of the balanced cut (i64: 2 + one per sequence)
+  p.order_bytes = align_up(((size_t)c->batch + 2) * sizeof(long long), 256);
   p.total_bytes = p.q_rot_bytes + p.part_o_bytes + p.part_ml_bytes + p.order_bytes;
   return p;
 }
@@ -222,7 +218,10 @@ int wedlm_window_attn(const wedlm_config_t* cfg, const void* q, const void* k, c
     rc = launch_attn_generic(s, plan, q_rot, k_cache, v_cache, block_table, prefix_len, out, part_o, part_ml, status, st);
   if (ev1 && cudaEventRecord(ev1, st) != cudaSuccess) return WEDLM_ERR_CUDA;
   if (rc != WEDLM_OK) return rc;
-  if (plan.n_splits > 1) rc = launch_attn_merge(s, plan, prefix_len, part_o, part_ml, out, st);
+  if (plan.impl == WEDLM_ATTN_TENSOR)
+    rc = launch_attn_tensor_merge(s, plan, prefix_len, order, part_o, part_ml, out, st);
+  else if (plan.n_splits > 1)
+    rc = launch_attn_merge(s, plan, prefix_len, part_o, part_ml, out, st);
   return rc;
 }
 

@@ -72,8 +72,10 @@ int launch_rope_stage(const Shape& s, const void* q, const void* k, const void* 
 
 struct AttnPlan {
   int impl;            // WEDLM_ATTN_GENERIC or WEDLM_ATTN_TENSOR
-  int n_splits;        // key chunks per (sequence, head)
-  int chunk;           // keys per chunk (multiple of the page size)
+  int n_splits;        // partial slots per query row: key chunks per (sequence, head), or pieces per unit (balanced)
+  int chunk;           // keys per chunk (multiple of the page size; CUDA-core path)
+  int balanced;        // tensor path with fewer work units than CTA slots: the tiles are cut into equal runs
+  int n_ctas;          // CTAs of the balanced cut
   size_t q_rot_bytes, part_o_bytes, part_ml_bytes, order_bytes, total_bytes;
 };
 AttnPlan plan_attention(const wedlm_config_t* cfg);
@@ -87,6 +89,9 @@ int launch_attn_tensor(const Shape& s, const AttnPlan& plan, const void* q_rot, 
                        const void* v_cache, const int32_t* block_table, const int32_t* prefix_len,
                        const int32_t* order, void* out, float* part_o, float* part_ml, int32_t* status,
                        cudaStream_t st);
+
+int launch_attn_tensor_merge(const Shape& s, const AttnPlan& plan, const int32_t* prefix_len, const int32_t* order,
+                             const float* part_o, const float* part_ml, void* out, cudaStream_t st);
 
 int launch_wait_expiry_selftest(uint32_t max_polls, int32_t* status, cudaStream_t st);
 

@@ -93,6 +93,18 @@ def test_large_windows(W):
     pu.full_parity(cfg, inp, attn_impl="generic" if W > 128 else "tensor")
 
 
+def test_long_ragged_sequences_whose_runs_cross_from_one_key_stream_into_the_next():
+    """Few work units and long prefixes: the tensor path cuts the key tiles of all (sequence, KV head) streams into
+    equal runs, here of about 35 tiles, so most CTAs finish one stream and start the next (another head, or another
+    sequence of different length), with two row tiles per stream sharing every run."""
+    import parity_util as pu
+    cfg = _small_qwen(batch=3, window=48, n_q_heads=8, n_kv_heads=2, prefix_lo=50000, prefix_hi=60000, vocab=512,
+                      name="crossing")
+    inp = make_step(cfg, seed=4848, prefix_len=np.array([60000, 50003, 55017], dtype=np.int32))
+    res = pu.full_parity(cfg, inp, attn_impl="tensor")
+    assert int(res["step"].status.item()) == 0
+
+
 @pytest.mark.parametrize("P", [0, 1, 15, 16, 17, 31, 33])
 def test_page_boundaries(P):
     import parity_util as pu
