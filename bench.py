@@ -30,10 +30,11 @@ UNIT = "tokens/s"
 L2_BYTES = 126 * 1024 * 1024
 
 # DRAM traffic of the dominant kernel as a multiple of its algorithmic bytes
-# (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture on a batch-16 case of the same
-# shapes; profiles/attn_tensor_kernel_cfg3_batch16.md gives the command).  Traffic grows with the
-# tokens streamed, so the ratio is applied to the launch that is timed.  Missing = not captured.
-NCU_TRAFFIC_RATIO = {"cfg3_batched:auto": 1.011, "cfg3_batched:tensor": 1.011}
+# (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture on a batch-40 case of the same
+# shapes, which runs the same one-unit-per-CTA scheduling as the full batch: 705.5 MB against 704.0 MB;
+# profiles/attn_tensor_kernel_cfg3_batch40.md gives the command).  Traffic grows with the tokens
+# streamed, so the ratio is applied to the launch that is timed.  Missing = not captured.
+NCU_TRAFFIC_RATIO = {"cfg3_batched:auto": 1.002, "cfg3_batched:tensor": 1.002}
 
 
 def log(*a):
@@ -600,7 +601,7 @@ def run_product(args):
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                          "frac_of_nominal_8TBps": achieved / 8000.0,
                          "traffic": (NCU_TRAFFIC_RATIO[key] * bts["attn_kernel"] if key in NCU_TRAFFIC_RATIO and not args.batch else None),
-                         "traffic_note": "ncu dram bytes of a batch-16 capture scaled by algorithmic bytes",
+                         "traffic_note": "ncu dram bytes of a batch-40 capture scaled by algorithmic bytes",
                          "kernel_ms": attn_ms,
                          "algorithmic_bytes": bts["attn_kernel"],
                          "bytes_definition": "K and V of every cached prefix token AND of the staged window rows (4096 B per token), "
@@ -709,7 +710,8 @@ def measure_loop(args):
             on_target = sum(int(out["y"][bb] == pt["target"][bb, P:P + N].tolist()) for bb in range(B))
             results.append({"window": W, "commit": mode, "lm_head": "fused" if fused else "gemm+logits",
                             "replay": "eager" if args.loop_eager else "cuda_graph",
-                            "tilt": f"{tilt_name}+{tilt:g}", "tokens_per_s": n_gen / dt, "seconds": dt,
+                            "tilt": f"{tilt_name}+{tilt:g}", "tokens_per_s": n_gen / out.get("decode_s", dt), "seconds": dt,
+                            "decode_seconds": out.get("decode_s", dt), "capture_seconds": out.get("capture_s", 0.0),
                             "steps": out["steps"], "tokens_per_step_per_seq": n_gen / B / max(out["steps"], 1),
                             "p_cache": out["p_cache"], "sequences_equal_to_target": on_target})
             log(results[-1])
@@ -719,7 +721,7 @@ def measure_loop(args):
             "config": {"workload": "cfg5_loop", "batch": B, "prompt": P, "new_tokens": N, "layers": m.n_layers,
                        "tau": args.loop_tau, "lambda": args.loop_lambda,
                        "hidden": H, "lse_of_untilted_logits": lse0,
-                       "timing": "host wall clock around generate(), after one short untimed run of the same geometry; includes the graph capture and the per-step read-back of commits"},
+                       "timing": "host wall clock of the decode loop (graph replays with the per-step read-back of commits), after one short untimed run of the same geometry; capturing the step once is timed apart (capture_seconds); eager runs time generate() whole"},
             "results": results}
     del wts, lm_head_vh
     return line

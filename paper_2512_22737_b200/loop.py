@@ -227,8 +227,13 @@ class StreamingDecoder:
                     commits_per_step=commits_per_step)
 
     def _generate_graph(self, max_new_tokens: int, max_steps: int) -> Dict[str, object]:
+        import time
         self.start(max_new_tokens)
+        t_capture = time.perf_counter()
         graph = self.capture_step()
+        torch.cuda.synchronize()
+        t_decode = time.perf_counter()
+        t_capture = t_decode - t_capture
         s = self.step_bufs
         B, W = self.B, self.W
         # one pinned buffer receives everything the host needs from a step: window_len | count | tokens
@@ -253,5 +258,7 @@ class StreamingDecoder:
                 ys[b].extend(ct_h[b, : cc_h[b]].tolist())
             commits_per_step.append(int(cc_h.sum()))
         n_gen = sum(len(y) for y in ys)
+        t_decode = time.perf_counter() - t_decode
+        # capture_s: capturing the step once; decode_s: the replay loop with its per-step read-back (host wall clock)
         return dict(y=ys, steps=self.steps, n_fwd=self.n_fwd, p_cache=(n_gen / self.n_fwd if self.n_fwd else 0.0),
-                    commits_per_step=commits_per_step)
+                    commits_per_step=commits_per_step, capture_s=t_capture, decode_s=t_decode)
