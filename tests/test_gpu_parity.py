@@ -105,6 +105,17 @@ def test_long_ragged_sequences_whose_runs_cross_from_one_key_stream_into_the_nex
     assert int(res["step"].status.item()) == 0
 
 
+def test_one_long_sequence_is_spread_over_every_cta_slot():
+    """A single sequence of 150 000 cached tokens: its 8 key streams are cut into about 37 pieces each (close to the
+    number of partial slots the workspace provides per row), one run per CTA slot, runs crossing from one KV head
+    into the next."""
+    import parity_util as pu
+    cfg = _small_qwen(batch=1, window=16, prefix_lo=150000, prefix_hi=150000, vocab=512, name="one_long")
+    inp = make_step(cfg, seed=150)
+    res = pu.full_parity(cfg, inp, attn_impl="tensor")
+    assert int(res["step"].status.item()) == 0
+
+
 @pytest.mark.parametrize("P", [0, 1, 15, 16, 17, 31, 33])
 def test_page_boundaries(P):
     import parity_util as pu
