@@ -38,6 +38,8 @@
  *     addresses.  Index tensors are int32, flags are uint8.
  *   - "logical order" = ascending position id within the window; "physical order" = the order
  *     after wedlm_reorder.  Slot j (logical) of sequence b has position id prefix_len[b] + j.
+ *   - Every call that launches work opens an NVTX range with its own name for its duration on the host
+ *     (a no-op unless a timeline tool is attached).
  *   - Return value: WEDLM_OK or a negative WEDLM_ERR_* code.  Argument errors are detected on
  *     the host before anything is launched.  Data-dependent errors (a block-table entry outside
  *     the page pool) are detected on the device: the offending access is skipped and a bit is

@@ -169,6 +169,7 @@ int wedlm_profile_next_attn(void* event_before, void* event_after) {
 int wedlm_reorder(const wedlm_config_t* cfg, const uint8_t* filled, const int32_t* window_tokens,
                   const int32_t* prefix_len, const int32_t* window_len, int32_t* perm, int32_t* inv_perm,
                   int32_t* pos_ids, int32_t* tokens_phys, int32_t* n_filled, int32_t* n_commit, void* stream) {
+  ApiRange nvtx_range("wedlm_reorder");
   int rc = check_config(cfg, false, false);
   if (rc != WEDLM_OK) return rc;
   if (cfg->batch == 0) return WEDLM_OK;
@@ -188,6 +189,7 @@ int wedlm_window_attn(const wedlm_config_t* cfg, const void* q, const void* k, c
                       void* v_cache, const int32_t* block_table, const int32_t* prefix_len, const int32_t* pos_ids,
                       void* out, int32_t* kv_slot_idx, void* workspace, size_t workspace_bytes, int32_t* status,
                       void* stream) {
+  ApiRange nvtx_range("wedlm_window_attn");
   int rc = check_config(cfg, true, false);
   if (rc != WEDLM_OK) return rc;
   if (cfg->batch == 0) return WEDLM_OK;
@@ -228,6 +230,7 @@ int wedlm_window_attn(const wedlm_config_t* cfg, const void* q, const void* k, c
 int wedlm_kv_append(const wedlm_config_t* cfg, const void* k, const void* v, const int32_t* pos_ids, void* k_cache,
                     void* v_cache, const int32_t* block_table, const int32_t* prefix_len, const int32_t* count,
                     int32_t* kv_slot_idx, int32_t* status, void* stream) {
+  ApiRange nvtx_range("wedlm_kv_append");
   int rc = check_config(cfg, true, false);
   if (rc != WEDLM_OK) return rc;
   if (cfg->batch == 0) return WEDLM_OK;
@@ -249,6 +252,7 @@ int wedlm_confidence_commit(const wedlm_config_t* cfg, const void* logits, const
                             int32_t* argmax, float* maxprob, float* entropy, float* lse, int32_t* committed_tokens,
                             int32_t* committed_count, int32_t* filled_count, void* workspace, size_t workspace_bytes,
                             int32_t* status, void* stream) {
+  ApiRange nvtx_range("wedlm_confidence_commit");
   int rc = check_config(cfg, false, true);
   if (rc != WEDLM_OK) return rc;
   if (cfg->batch == 0) return WEDLM_OK;
@@ -273,6 +277,7 @@ int wedlm_lmhead_confidence_commit(const wedlm_config_t* cfg, int32_t hidden, co
                                    int32_t* argmax, float* maxprob, float* entropy, float* lse, int32_t* committed_tokens,
                                    int32_t* committed_count, int32_t* filled_count, void* workspace, size_t workspace_bytes,
                                    int32_t* status, void* stream) {
+  ApiRange nvtx_range("wedlm_lmhead_confidence_commit");
   int rc = check_config(cfg, false, true);
   if (rc != WEDLM_OK) return rc;
   if (cfg->dtype != WEDLM_DTYPE_BF16 || hidden < 64 || hidden % 64 != 0) return WEDLM_ERR_UNSUPPORTED;
@@ -337,6 +342,7 @@ int plan_dual_stream(const wedlm_config_t* cfg, int32_t n_blocks, DualPlan* out)
 int wedlm_dual_stream_construct(const wedlm_config_t* cfg, int32_t n_blocks, int32_t seq_len, const int32_t* tokens,
                                 const uint8_t* masked, int32_t* x_input, int32_t* p_input, uint8_t* is_mask,
                                 int32_t* n_observed, void* stream) {
+  ApiRange nvtx_range("wedlm_dual_stream_construct");
   if (cfg == nullptr || n_blocks < 1 || cfg->batch < 0 || cfg->window < 1 || cfg->window > 1024) return WEDLM_ERR_INVALID_ARG;
   if (seq_len < 1 || (long long)seq_len > (long long)n_blocks * cfg->window ||
       (long long)seq_len <= (long long)(n_blocks - 1) * cfg->window)
@@ -357,6 +363,7 @@ size_t wedlm_dual_stream_workspace_bytes(const wedlm_config_t* cfg, int32_t n_bl
 int wedlm_dual_stream_attn(const wedlm_config_t* cfg, int32_t n_blocks, const void* q, const void* k, const void* v,
                            const int32_t* p_input, void* out, void* workspace, size_t workspace_bytes, int32_t* status,
                            void* stream) {
+  ApiRange nvtx_range("wedlm_dual_stream_attn");
   DualPlan p;
   int rc = plan_dual_stream(cfg, n_blocks, &p);
   if (rc != WEDLM_OK) return rc;
@@ -608,6 +615,7 @@ int wedlm_step_host(const wedlm_config_t* cfg, uint8_t* h_filled, int32_t* h_win
                     const void* h_k, const void* h_v, const void* h_logits, void* k_cache, void* v_cache,
                     int32_t* h_committed_tokens, int32_t* h_committed_count, int32_t* h_filled_count, void* workspace,
                     size_t workspace_bytes, void** attn_out, int32_t* status, void* stream) {
+  ApiRange nvtx_range("wedlm_step_host");
   return step_host_impl(cfg, 0, h_filled, h_window_tokens, h_prefix_len, h_window_len, h_remaining_budget, h_block_table, h_q,
                         h_k, h_v, h_logits, nullptr, nullptr, nullptr, 0.f, k_cache, v_cache, h_committed_tokens,
                         h_committed_count, h_filled_count, workspace, workspace_bytes, attn_out, status, stream);
@@ -620,6 +628,7 @@ int wedlm_step_host_lmhead(const wedlm_config_t* cfg, int32_t hidden, uint8_t* h
                            void* k_cache, void* v_cache, int32_t* h_committed_tokens, int32_t* h_committed_count,
                            int32_t* h_filled_count, void* workspace, size_t workspace_bytes, void** attn_out,
                            int32_t* status, void* stream) {
+  ApiRange nvtx_range("wedlm_step_host_lmhead");
   if (cfg == nullptr || cfg->dtype != WEDLM_DTYPE_BF16 || hidden < 64 || hidden % 64 != 0) return WEDLM_ERR_UNSUPPORTED;
   return step_host_impl(cfg, hidden, h_filled, h_window_tokens, h_prefix_len, h_window_len, h_remaining_budget, h_block_table,
                         h_q, h_k, h_v, nullptr, h_hidden_states, lm_head, h_tilt_ids, tilt, k_cache, v_cache,
@@ -630,6 +639,7 @@ int wedlm_step_host_lmhead(const wedlm_config_t* cfg, int32_t hidden, uint8_t* h
 int wedlm_window_refill(const wedlm_config_t* cfg, const int32_t* n_commit, int32_t* window_tokens, uint8_t* filled,
                         int32_t* prefix_len, int32_t* window_len, int32_t* remaining_budget,
                         int32_t* committed_tokens, int32_t* committed_count, void* stream) {
+  ApiRange nvtx_range("wedlm_window_refill");
   int rc = check_config(cfg, false, false);
   if (rc != WEDLM_OK) return rc;
   if (cfg->batch == 0) return WEDLM_OK;

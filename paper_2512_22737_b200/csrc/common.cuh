@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "wedlm.h"
 
 namespace wedlm {
@@ -141,5 +143,13 @@ int device_sm_count();
 
 // Number of kernels this process has launched through the library (reported by wedlm_launch_count).
 void count_launch(int n = 1);
+
+// NVTX range around a public call: shows up by name in a timeline tool, costs nothing without one attached.
+struct ApiRange {
+  explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+  ~ApiRange() { nvtxRangePop(); }
+  ApiRange(const ApiRange&) = delete;
+  ApiRange& operator=(const ApiRange&) = delete;
+};
 
 }  // namespace wedlm

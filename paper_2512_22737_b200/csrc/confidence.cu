@@ -864,6 +864,7 @@ extern "C" int wedlm_confidence_commit_static(const wedlm_config_t* cfg, const v
                                               float* maxprob, float* entropy, float* lse,
                                               int32_t* committed_tokens, int32_t* committed_count,
                                               int32_t* filled_count, int32_t* status, void* stream) {
+  wedlm::ApiRange nvtx_range("wedlm_confidence_commit_static");
   const size_t need = wedlm_confidence_workspace_bytes(cfg);     // 0 for a NULL / invalid config
   if (need == 0) return WEDLM_ERR_INVALID_ARG;
   if (need > (size_t)WEDLM_STATIC_SCRATCH_BYTES) return WEDLM_ERR_STATIC_SCRATCH;
