@@ -623,11 +623,20 @@ attn_merge_balanced_kernel(const TensorAttnParams p) {
     for (int o = 16; o > 0; o >>= 1) lw += __shfl_xor_sync(0xffffffffu, lw, o);
     l += lw;
     const int n_here = min(32, n_pieces - base);
-    for (int sp = 0; sp < n_here; ++sp) {
-      const float ws = __shfl_sync(0xffffffffu, wgt, sp);
-      if (ws == 0.f) continue;
-      const float4 o = *reinterpret_cast<const float4*>(p.part_o + (prow + base + sp) * kD + d);
-      acc.x += ws * o.x; acc.y += ws * o.y; acc.z += ws * o.z; acc.w += ws * o.w;
+    for (int sp0 = 0; sp0 < n_here; sp0 += 4) {          // four pieces at a time, so that their loads overlap
+      float ws[4];
+      float4 o[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        ws[u] = __shfl_sync(0xffffffffu, wgt, (sp0 + u) & 31);
+        if (sp0 + u >= n_here) ws[u] = 0.f;
+        o[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ws[u] != 0.f) o[u] = *reinterpret_cast<const float4*>(p.part_o + (prow + base + sp0 + u) * kD + d);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        acc.x += ws[u] * o[u].x; acc.y += ws[u] * o[u].y; acc.z += ws[u] * o[u].z; acc.w += ws[u] * o[u].w;
+      }
     }
   }
   const float inv = l > 0.f ? 1.f / l : 0.f;
