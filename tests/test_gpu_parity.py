@@ -93,6 +93,18 @@ def test_large_windows(W):
     pu.full_parity(cfg, inp, attn_impl="generic" if W > 128 else "tensor")
 
 
+@pytest.mark.parametrize("W,P", [(512, 700), (1024, 3000)])
+def test_many_row_tiles_share_the_runs_of_one_key_stream(W, P):
+    """Tensor path with 16 and 32 row tiles per key stream: every run of key tiles is taken by one CTA per row tile,
+    and the row tiles of the early window slots, whose horizon ends sooner, skip the last runs."""
+    import parity_util as pu
+    cfg = _small_qwen(batch=2, window=W, n_q_heads=4, n_kv_heads=1, prefix_lo=P, prefix_hi=P + 200, vocab=512,
+                      name="manytiles")
+    inp = make_step(cfg, seed=W + P)
+    res = pu.full_parity(cfg, inp, attn_impl="tensor")
+    assert int(res["step"].status.item()) == 0
+
+
 def test_long_ragged_sequences_whose_runs_cross_from_one_key_stream_into_the_next():
     """Few work units and long prefixes: the tensor path cuts the key tiles of all (sequence, KV head) streams into
     equal runs, here of about 35 tiles, so most CTAs finish one stream and start the next (another head, or another
