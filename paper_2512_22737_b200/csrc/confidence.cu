@@ -185,12 +185,14 @@ conf_partial_kernel(int W, int V, int n_chunks, const T* __restrict__ logits, co
 
 // ------------------------------------------------------------------------------------------------
 // Streaming variant of pass 1 for bf16 logits with 16-byte aligned rows: persistent blocks pull
-// (row, chunk) items of active mask rows through a 4-stage shared-memory ring filled by bulk
-// asynchronous copies (one 16 KB copy per item, completion on an mbarrier), so that the bytes in
-// flight per SM do not depend on registers.  Same chunking and partial layout as conf_partial_kernel.
+// (row, chunk) items of active mask rows through a shared-memory slot filled by bulk asynchronous
+// copies (one 16 KB copy per item, completion on an mbarrier).  The consumers move an item into
+// registers at once and hand the slot back, so one slot per block is enough to keep a copy in
+// flight while they compute, and eight blocks fit on an SM (48 registers, 16 KB).  Same chunking and
+// partial layout as conf_partial_kernel.
 // ------------------------------------------------------------------------------------------------
-constexpr int kStreamStages = 2;                                    // power of two (stage = n & (stages - 1))
-constexpr int kStreamBlocksPerSM = 6;                               // 32 KB ring each
+constexpr int kStreamStages = 1;                                    // slots per block; power of two (slot = n & (stages - 1))
+constexpr int kStreamBlocksPerSM = 8;                               // two 16 KB slots and 6 blocks measured 2 % slower
 constexpr int kStreamThreads = 128;                                 // consumer threads per block
 constexpr int kStreamVecs = 8;                                      // 16-byte vectors per thread and item
 constexpr int kStreamChunk = kStreamThreads * kStreamVecs * 8;      // 8192 bf16 = 16 KB, same chunking as pass 1 above
@@ -217,7 +219,7 @@ __device__ __forceinline__ void cs_consumer_sync() {     // the consumer threads
 }
 
 // block = 4 consumer warps + 1 producer warp (its lane 0 issues the copies)
-__global__ void __launch_bounds__(kStreamThreads + 32)
+__global__ void __launch_bounds__(kStreamThreads + 32, kStreamBlocksPerSM)
 conf_stream_kernel(int W, int V, int n_chunks, long long total_items, const __nv_bfloat16* __restrict__ logits,
                    const int32_t* __restrict__ n_filled, const int32_t* __restrict__ window_len,
                    float4* __restrict__ part, int32_t* status) {
