@@ -627,13 +627,14 @@ def run_product(args):
 # ----------------------------------------------------------------------------------------------
 def measure_loop_short(args):
     """The end-to-end loop in a form short enough for the default line: 256 new tokens per sequence at the
-    calibrated tilt lse + 8, streaming commits, W = 16 against the same harness at W = 2 and W = 1."""
+    calibrated tilt lse + 8, streaming commits, W = 16 against the same harness at W = 2 and W = 1, and W = 16 once
+    more with the LM head fused into the confidence call."""
     import types
     a = types.SimpleNamespace(**vars(args))
-    a.loop_new_tokens, a.loop_windows, a.loop_block_windows, a.loop_fused_windows = 256, [16, 2, 1], [], []
+    a.loop_new_tokens, a.loop_windows, a.loop_block_windows, a.loop_fused_windows = 256, [16, 2, 1], [], [16]
     a.loop_tilts, a.loop_eager = [("lse", 8.0)], False
     line = measure_loop(a)
-    by_w = {r["window"]: r for r in line["results"]}
+    by_w = {r["window"]: r for r in line["results"] if r["lm_head"] != "fused"}
     out = {"config": line["config"], "results": line["results"], "unit": "generated tokens/s"}
     if 16 in by_w and 1 in by_w:
         out["speedup_w16_over_w1"] = by_w[16]["tokens_per_s"] / by_w[1]["tokens_per_s"]

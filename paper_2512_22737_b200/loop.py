@@ -60,7 +60,7 @@ class StreamingDecoder:
         if fused_lm_head:
             if "lm_head" in self.wt:
                 self.lm_head_vh = self.wt["lm_head"].t().contiguous()
-            self.lm_ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(self.cfg, int(self.wt["embed"].shape[1])), dtype=torch.uint8, device="cuda")
+            self.lm_ws = torch.empty(w.wedlm_lmhead_confidence_workspace_bytes(self.cfg, int(mcfg.hidden)), dtype=torch.uint8, device="cuda")
         i32 = dict(dtype=torch.int32, device="cuda")
         self.window_tokens = torch.full((batch, window), mcfg.mask_token_id, **i32)
         self.filled = torch.zeros(batch, window, dtype=torch.uint8, device="cuda")
